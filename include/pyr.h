@@ -1,0 +1,212 @@
+/*
+ * pyr.h - C ABI of the PyramidInfer prefill-selection hot path for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library implements one layer-wise step of PyramidInfer (arXiv
+ * 2405.12532, Algorithm 1, prefill branch, and the attention of the generation
+ * phase of Section 4.1):
+ *
+ *   pyr_prefill_layer   attention weights over the tokens the layer received,
+ *                       the attention output, and the ensemble score A_e that
+ *                       the most recent L queries give every context key;
+ *   pyr_select_compact  TopP index (a count-based top-k) + Gather: K/V of the
+ *                       kept keys go to the layer's cache, rows that feed the
+ *                       next layer are compacted in place;
+ *   pyr_decode_attn     one generation step of one layer over its compressed,
+ *                       per-layer-sized cache;
+ *   pyr_cache_alloc     the pyramid itself: per-layer budgets from the ratio
+ *                       schedule and the cache carved out of caller memory.
+ *
+ * Conventions
+ *   - Plain C. Every call returns a pyr_status_t, never throws, aborts or
+ *     prints.
+ *   - Pointers marked "device" are caller-owned device memory that must stay
+ *     valid until the stream work that uses them has finished. Pointers marked
+ *     "host" are read (or written) before the call returns.
+ *   - The library allocates no device memory: the caller passes one buffer of
+ *     pyr_cache_bytes() bytes. Only the host-side handle is library-owned.
+ *   - Every launching call takes a CUDA stream (cudaStream_t passed as void*,
+ *     NULL = the default stream), enqueues its kernels there and returns; it
+ *     does not synchronise. All shapes follow from the schedule on the host,
+ *     so nothing is copied back.
+ *   - A device-side wait that runs out (bounded spin on an mbarrier) records a
+ *     code in a device status word and the kernel returns; read it with
+ *     pyr_cache_status().
+ *   - A handle is not thread-safe; use one per thread or lock around it.
+ *
+ * Tensor layouts (element = bf16 or fp32 as configured, D = head_dim innermost
+ * and contiguous)
+ *   q, out        [B, n, Hq,  D]   strides given in elements
+ *   k, v          [B, n, Hkv, D]   strides given in elements
+ *   layer cache   [B, Hkv, cap_l, D] for K and for V
+ *   scores        [B, G, c]  fp32, G = sel_groups, c = n - L context keys
+ *   lse           [B, Hq, n] fp32, natural log of the softmax denominator
+ *   kept / pos    [B, G, n_out] int32
+ */
+#ifndef PYR_H_
+#define PYR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PYR_OK = 0,
+  PYR_ERR_INVALID = 1,          /* a value outside its documented range            */
+  PYR_ERR_NULL = 2,             /* a required pointer is NULL                      */
+  PYR_ERR_UNSUPPORTED = 3,      /* dtype / head_dim / size / device not supported  */
+  PYR_ERR_BUFFER_TOO_SMALL = 4, /* dev_buf smaller than pyr_cache_bytes()          */
+  PYR_ERR_CAPACITY = 5,         /* decode append beyond max_new_tokens             */
+  PYR_ERR_ORDER = 6,            /* call out of the prefill/select/decode sequence  */
+  PYR_ERR_CUDA = 7,             /* a CUDA runtime call failed                      */
+  PYR_ERR_TIMEOUT = 8           /* a bounded device-side wait ran out              */
+} pyr_status_t;
+
+typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
+
+/* flags */
+#define PYR_FLAG_CUDA_CORE_PREFILL 1u /* bf16 prefill on the CUDA-core kernel (validation aid) */
+
+/*
+ * Parameters of Algorithm 1 (recent window length L, minimum PvC lengths N_l,
+ * ratio p and its decay, given here as one explicit ratio per layer) plus the
+ * attention geometry.
+ */
+typedef struct {
+  int32_t n_layers;
+  int32_t n_q_heads;      /* Hq                                                        */
+  int32_t n_kv_heads;     /* Hkv, divides Hq                                           */
+  int32_t head_dim;       /* D: 64 or 128                                              */
+  int32_t sel_groups;     /* G: 1 (one kept set per sequence) or Hkv (one per KV head) */
+  int32_t dtype;          /* pyr_dtype_t of q/k/v/out and of the cache                 */
+  int32_t batch;          /* B                                                         */
+  int32_t prompt_len;     /* N, the same for every sequence of the batch               */
+  int32_t recent_len;     /* L >= 1: the recent window S_r, never evicted              */
+  int32_t max_new_tokens; /* T: rows reserved per layer for decode appends             */
+  const double* ratio;    /* host [n_layers]: fraction of the ORIGINAL context
+                             c_0 = N - L that layer l keeps; each in [0,1],
+                             non-increasing                                            */
+  const int32_t* min_len; /* host [n_layers] or NULL: N_l, lower bound on the kept
+                             length (window included) of layer l                       */
+  const float* recent_w;  /* host [L] or NULL: non-negative weights of the recent
+                             queries, oldest first. NULL = linear ramp
+                             2(i+1)/(L(L+1)), which sums to 1                          */
+  float softmax_scale;    /* 0 = 1/sqrt(D)                                             */
+  uint32_t flags;
+} pyr_config_t;
+
+typedef struct pyr_cache pyr_cache_t;
+
+/* Algorithm 1's schedule (p, decay, N_l) as integers: for layer `layer` the
+ * tokens it receives (n_in), the context keys it keeps (k_ctx; the kept length
+ * is k_ctx + min(L, n_in)), the rows now in its cache (len_now) and the cache
+ * capacity in rows (cap). k_ctx = min(c, max(floor(ratio*c_0), N_l - L, 0)).
+ * Host arithmetic only; any out pointer may be NULL. */
+pyr_status_t pyr_cache_layer_info(const pyr_cache_t* cache, int32_t layer, int32_t* n_in,
+                                  int32_t* k_ctx, int32_t* len_now, int32_t* cap);
+
+/* Size and alignment of the device buffer pyr_cache_alloc needs for `cfg`
+ * (Section 4.1: each layer's cache holds only its PvC and window, plus T
+ * decode rows; the buffer also holds scores, lse, kept indices, positions, the
+ * decode workspace and the status word). Validates cfg. */
+pyr_status_t pyr_cache_bytes(const pyr_config_t* cfg, size_t* bytes, size_t* align);
+
+/* Builds a cache handle over the caller's device buffer `dev_buf` (device,
+ * `bytes` long, aligned as pyr_cache_bytes says). Copies cfg and its arrays.
+ * Touches no device memory and makes no CUDA call. *out is set on PYR_OK. */
+pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t bytes,
+                             pyr_cache_t** out);
+
+/* Frees the host handle. The device buffer stays the caller's. */
+pyr_status_t pyr_cache_free(pyr_cache_t* cache);
+
+/* Starts a new prompt batch with the same configuration: layer 0's prefill is
+ * expected next; clears the device status word on `stream`. */
+pyr_status_t pyr_cache_reset(pyr_cache_t* cache, void* stream);
+
+/* Device pointers (valid until the next pyr_select_compact) to the kept indices
+ * [B, G, n_out] of `layer`'s selection - ascending positions within the layer's
+ * input, window last - and to the ORIGINAL prompt positions of those tokens
+ * (Appendix A.2, "gather" position encoding). `layer` must be the layer most
+ * recently selected. */
+pyr_status_t pyr_cache_kept(const pyr_cache_t* cache, int32_t layer, const int32_t** dev_idx,
+                            const int32_t** dev_pos);
+
+/* Device pointer to the pooled ensemble scores [B, G, c] that the most recent
+ * pyr_prefill_layer(layer) wrote (valid until the next prefill call). */
+pyr_status_t pyr_cache_scores(const pyr_cache_t* cache, int32_t layer, const float** dev_scores);
+
+/* Device pointer to lse [B, Hq, n_in] of the most recent pyr_prefill_layer. */
+pyr_status_t pyr_cache_lse(const pyr_cache_t* cache, int32_t layer, const float** dev_lse);
+
+/* Device pointers to layer `layer`'s K and V cache [B, Hkv, cap, D]. */
+pyr_status_t pyr_cache_kv(const pyr_cache_t* cache, int32_t layer, void** dev_k, void** dev_v);
+
+/* Synchronises `stream`, copies the device status word to *host_status
+ * (a pyr_status_t: PYR_OK or PYR_ERR_TIMEOUT) and returns it. */
+pyr_status_t pyr_cache_status(pyr_cache_t* cache, void* stream, int32_t* host_status);
+
+/*
+ * Algorithm 1, "compute attention weights of KV" and
+ * "A_e <- weighted_avg(A[-L:, :-L], dim=-2)" for one layer.
+ *
+ * q, k, v (device) hold the layer's n_in tokens in ascending original order.
+ * Writes out = softmax(scale q k^T + causal mask) v for all n_in rows, lse into
+ * the cache, and the pooled score
+ *     score[b,g,j] = mean over the query heads h of group g of
+ *                    sum_i w_i * A_h[c+i, j],   j < c = n_in - L,
+ * into the cache. The L x c block of weights is never stored. Layers must be
+ * called in order, each followed by pyr_select_compact (PYR_ERR_ORDER
+ * otherwise). Strides are in elements; the innermost (D) stride is 1. For
+ * bf16 the base pointers and strides must keep every row 16-byte aligned.
+ */
+pyr_status_t pyr_prefill_layer(pyr_cache_t* cache, int32_t layer, const void* q, const void* k,
+                               const void* v, void* out, int64_t q_stride_b, int64_t q_stride_n,
+                               int64_t q_stride_h, int64_t kv_stride_b, int64_t kv_stride_n,
+                               int64_t kv_stride_h, int64_t o_stride_b, int64_t o_stride_n,
+                               int64_t o_stride_h, void* stream);
+
+/*
+ * Algorithm 1, "TopP_index <- TopP(A_e, p)" and "PvC <- Gather(KV, TopP_index)".
+ *
+ * Per (sequence, selection group): the k_ctx largest scores left by
+ * pyr_prefill_layer(layer) are kept, an exact tie going to the lower index;
+ * the kept list is those keys in ascending order followed by the whole window.
+ * K and V (device, the same tensors the prefill call read) are gathered into
+ * the layer's cache. `rows` (device, may be NULL) is compacted IN PLACE to the
+ * kept rows: row i of the result is former row kept[i]. With sel_groups == 1,
+ * rows is [B, n_in, row_elems] (rows_stride_g must be 0), e.g. hidden states;
+ * with sel_groups == Hkv it is addressed as
+ * rows + b*rows_stride_b + g*rows_stride_g + i*rows_stride_n, row_elems
+ * contiguous elements per row, e.g. the attention output of the group's heads.
+ * Position ids are compacted alongside. *n_out (host, may be NULL) receives
+ * k_ctx + window. Dropped rows are neither read nor written.
+ */
+pyr_status_t pyr_select_compact(pyr_cache_t* cache, int32_t layer, const void* k, const void* v,
+                                int64_t kv_stride_b, int64_t kv_stride_n, int64_t kv_stride_h,
+                                void* rows, int64_t row_elems, int64_t rows_stride_b,
+                                int64_t rows_stride_n, int64_t rows_stride_g, int32_t* n_out,
+                                void* stream);
+
+/*
+ * Section 4.1, generation phase: the new token's key and value (device,
+ * [B, Hkv, D] contiguous) are appended to layer `layer`'s cache, then q
+ * (device, [B, Hq, D] contiguous) attends over all len_now + 1 rows, unmasked.
+ * out (device, [B, Hq, D]). Allowed once every layer has been selected.
+ * PYR_ERR_CAPACITY when the layer already holds cap rows.
+ */
+pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, const void* k_new,
+                             const void* v_new, void* out, void* stream);
+
+const char* pyr_status_string(pyr_status_t status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int32_t pyr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PYR_H_ */

@@ -1,0 +1,405 @@
+// Host side of the C ABI: argument validation, the pyramid schedule
+// (Algorithm 1: ratio p per layer, minimum PvC lengths N_l), carving of the
+// caller's device buffer, call ordering, and dispatch to the kernels.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "pyr_internal.h"
+
+namespace {
+
+struct LayerPlan {
+  int n_in, c, k, n_out, cap;
+  size_t k_off, v_off;   // byte offsets into the device buffer
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+constexpr size_t kAlign = 256;
+
+struct Layout {
+  size_t status, w, score, lse, idx, pos0, pos1, part_acc, part_ml, total;
+  std::vector<LayerPlan> layers;
+};
+
+pyr_status_t validate(const pyr_config_t* c) {
+  if (!c) return PYR_ERR_NULL;
+  if (!c->ratio) return PYR_ERR_NULL;
+  if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->batch < 1 ||
+      c->prompt_len < 1 || c->recent_len < 1 || c->max_new_tokens < 0)
+    return PYR_ERR_INVALID;
+  if (c->n_q_heads % c->n_kv_heads != 0) return PYR_ERR_INVALID;
+  if (c->sel_groups != 1 && c->sel_groups != c->n_kv_heads) return PYR_ERR_INVALID;
+  if (c->dtype != PYR_BF16 && c->dtype != PYR_F32) return PYR_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return PYR_ERR_UNSUPPORTED;
+  if (c->prompt_len > pyr::kMaxPrompt) return PYR_ERR_UNSUPPORTED;
+  if (!(c->softmax_scale >= 0.0f) || !std::isfinite(c->softmax_scale)) return PYR_ERR_INVALID;
+  double prev = 1.0;
+  for (int l = 0; l < c->n_layers; ++l) {
+    double r = c->ratio[l];
+    if (!(r >= 0.0 && r <= 1.0)) return PYR_ERR_INVALID;
+    if (r > prev) return PYR_ERR_INVALID;
+    prev = r;
+    if (c->min_len && c->min_len[l] < 0) return PYR_ERR_INVALID;
+  }
+  if (c->recent_w) {
+    int L = c->recent_len;
+    for (int i = 0; i < L; ++i)
+      if (!(c->recent_w[i] >= 0.0f) || !std::isfinite(c->recent_w[i])) return PYR_ERR_INVALID;
+  }
+  return PYR_OK;
+}
+
+// Budgets: k_l = min(c, max(floor(ratio_l * c_0), N_l - L, 0)); the window is
+// never evicted; a layer with no context keeps everything.
+void plan(const pyr_config_t* c, Layout* lay) {
+  const int N = c->prompt_len, L = c->recent_len;
+  const int c0 = N > L ? N - L : 0;
+  const size_t eb = c->dtype == PYR_BF16 ? 2 : 4;
+  const size_t B = c->batch, G = c->sel_groups, Hq = c->n_q_heads, Hkv = c->n_kv_heads,
+               D = c->head_dim;
+  size_t off = 0;
+  lay->status = off; off = align_up(off + pyr::kStatusWords * sizeof(int), kAlign);
+  lay->w = off;      off = align_up(off + (size_t)L * 4, kAlign);
+  lay->score = off;  off = align_up(off + B * G * (size_t)(c0 > 0 ? c0 : 1) * 4, kAlign);
+  lay->lse = off;    off = align_up(off + B * Hq * (size_t)N * 4, kAlign);
+  lay->idx = off;    off = align_up(off + B * G * (size_t)N * 4, kAlign);
+  lay->pos0 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);
+  lay->pos1 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);
+  lay->part_acc = off;
+  if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * D * 4, kAlign);
+  lay->part_ml = off;
+  if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * 2 * 4, kAlign);
+  lay->layers.resize(c->n_layers);
+  int n_in = N;
+  for (int l = 0; l < c->n_layers; ++l) {
+    LayerPlan& p = lay->layers[l];
+    p.n_in = n_in;
+    p.c = n_in > L ? n_in - L : 0;
+    const int window = n_in - p.c;
+    long long want = (long long)std::floor(c->ratio[l] * (double)c0);
+    long long lo = c->min_len ? (long long)c->min_len[l] - L : 0;
+    long long k = want > lo ? want : lo;
+    if (k < 0) k = 0;
+    if (k > p.c) k = p.c;
+    p.k = (int)k;
+    p.n_out = p.k + window;
+    p.cap = p.n_out + c->max_new_tokens;
+    const size_t bytes = B * Hkv * (size_t)p.cap * D * eb;
+    p.k_off = off; off = align_up(off + bytes, kAlign);
+    p.v_off = off; off = align_up(off + bytes, kAlign);
+    n_in = p.n_out;
+  }
+  lay->total = off;
+}
+
+}  // namespace
+
+struct pyr_cache {
+  pyr_config_t cfg;
+  std::vector<double> ratio;
+  std::vector<int32_t> min_len;
+  std::vector<float> w;
+  Layout lay;
+  char* base;
+  std::vector<int> len_now;
+  int next_layer;     // layer whose prefill (phase 0) or select (phase 1) comes next
+  int phase;
+  int pos_cur;        // which of pos0/pos1 holds the positions of the last selection
+  int last_selected;  // layer of the last pyr_select_compact, -1 if none
+  int last_prefilled;
+  bool needs_init;
+  float scale;
+};
+
+namespace {
+
+template <class T>
+T* at(const pyr_cache* c, size_t off) { return reinterpret_cast<T*>(c->base + off); }
+
+pyr_status_t device_init(pyr_cache* c, cudaStream_t s) {
+  if (cudaMemsetAsync(at<int>(c, c->lay.status), 0, pyr::kStatusWords * sizeof(int), s) != cudaSuccess)
+    return PYR_ERR_CUDA;
+  if (c->needs_init) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PYR_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+      return PYR_ERR_CUDA;
+    if (major != 10) return PYR_ERR_UNSUPPORTED;
+    if (cudaMemcpyAsync(at<float>(c, c->lay.w), c->w.data(), c->w.size() * 4, cudaMemcpyHostToDevice,
+                        s) != cudaSuccess)
+      return PYR_ERR_CUDA;
+    c->needs_init = false;
+  }
+  return PYR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pyr_status_string(pyr_status_t s) {
+  switch (s) {
+    case PYR_OK: return "ok";
+    case PYR_ERR_INVALID: return "invalid argument";
+    case PYR_ERR_NULL: return "null pointer";
+    case PYR_ERR_UNSUPPORTED: return "unsupported dtype, head_dim, size or device";
+    case PYR_ERR_BUFFER_TOO_SMALL: return "device buffer too small";
+    case PYR_ERR_CAPACITY: return "layer cache is full";
+    case PYR_ERR_ORDER: return "call out of sequence";
+    case PYR_ERR_CUDA: return "CUDA runtime error";
+    case PYR_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int32_t pyr_version(void) { return 100; }
+
+pyr_status_t pyr_cache_bytes(const pyr_config_t* cfg, size_t* bytes, size_t* align) {
+  pyr_status_t st = validate(cfg);
+  if (st != PYR_OK) return st;
+  if (!bytes) return PYR_ERR_NULL;
+  Layout lay;
+  plan(cfg, &lay);
+  *bytes = lay.total;
+  if (align) *align = kAlign;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t bytes, pyr_cache_t** out) {
+  pyr_status_t st = validate(cfg);
+  if (st != PYR_OK) return st;
+  if (!dev_buf || !out) return PYR_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(dev_buf) % kAlign) return PYR_ERR_INVALID;
+  pyr_cache* c = new (std::nothrow) pyr_cache();
+  if (!c) return PYR_ERR_INVALID;
+  c->cfg = *cfg;
+  c->ratio.assign(cfg->ratio, cfg->ratio + cfg->n_layers);
+  if (cfg->min_len) c->min_len.assign(cfg->min_len, cfg->min_len + cfg->n_layers);
+  c->cfg.ratio = c->ratio.data();
+  c->cfg.min_len = cfg->min_len ? c->min_len.data() : nullptr;
+  const int L = cfg->recent_len;
+  c->w.resize(L);
+  for (int i = 0; i < L; ++i)
+    c->w[i] = cfg->recent_w ? cfg->recent_w[i]
+                            : (float)(2.0 * (i + 1.0) / ((double)L * (double)(L + 1)));
+  c->cfg.recent_w = c->w.data();
+  plan(&c->cfg, &c->lay);
+  if (bytes < c->lay.total) { delete c; return PYR_ERR_BUFFER_TOO_SMALL; }
+  c->base = static_cast<char*>(dev_buf);
+  c->len_now.assign(cfg->n_layers, 0);
+  c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
+  c->needs_init = true;
+  c->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
+  *out = c;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_free(pyr_cache_t* c) {
+  if (!c) return PYR_ERR_NULL;
+  delete c;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_reset(pyr_cache_t* c, void* stream) {
+  if (!c) return PYR_ERR_NULL;
+  c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
+  std::fill(c->len_now.begin(), c->len_now.end(), 0);
+  return device_init(c, static_cast<cudaStream_t>(stream));
+}
+
+pyr_status_t pyr_cache_layer_info(const pyr_cache_t* c, int32_t layer, int32_t* n_in, int32_t* k_ctx,
+                                  int32_t* len_now, int32_t* cap) {
+  if (!c) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  const LayerPlan& p = c->lay.layers[layer];
+  if (n_in) *n_in = p.n_in;
+  if (k_ctx) *k_ctx = p.k;
+  if (len_now) *len_now = c->len_now[layer];
+  if (cap) *cap = p.cap;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_kept(const pyr_cache_t* c, int32_t layer, const int32_t** dev_idx,
+                            const int32_t** dev_pos) {
+  if (!c) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (layer != c->last_selected) return PYR_ERR_ORDER;
+  if (dev_idx) *dev_idx = at<int32_t>(c, c->lay.idx);
+  if (dev_pos) *dev_pos = at<int32_t>(c, c->pos_cur ? c->lay.pos1 : c->lay.pos0);
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_scores(const pyr_cache_t* c, int32_t layer, const float** dev_scores) {
+  if (!c || !dev_scores) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (layer != c->last_prefilled) return PYR_ERR_ORDER;
+  *dev_scores = at<float>(c, c->lay.score);
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_lse(const pyr_cache_t* c, int32_t layer, const float** dev_lse) {
+  if (!c || !dev_lse) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (layer != c->last_prefilled) return PYR_ERR_ORDER;
+  *dev_lse = at<float>(c, c->lay.lse);
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_kv(const pyr_cache_t* c, int32_t layer, void** dev_k, void** dev_v) {
+  if (!c) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (dev_k) *dev_k = c->base + c->lay.layers[layer].k_off;
+  if (dev_v) *dev_v = c->base + c->lay.layers[layer].v_off;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_status(pyr_cache_t* c, void* stream, int32_t* host_status) {
+  if (!c || !host_status) return PYR_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, at<int>(c, c->lay.status), sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return PYR_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return PYR_ERR_CUDA;
+  *host_status = word;
+  return word == 0 ? PYR_OK : PYR_ERR_TIMEOUT;
+}
+
+pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, const void* k, const void* v,
+                               void* out, int64_t qsb, int64_t qsn, int64_t qsh, int64_t ksb, int64_t ksn,
+                               int64_t ksh, int64_t osb, int64_t osn, int64_t osh, void* stream) {
+  if (!c || !q || !k || !v || !out) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (layer != c->next_layer || c->phase != 0) return PYR_ERR_ORDER;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int D = c->cfg.head_dim;
+  if (qsh < D || ksh < D || osh < D || qsn < D || ksn < D || osn < D) return PYR_ERR_INVALID;
+  if (c->cfg.dtype == PYR_BF16) {
+    const uintptr_t m = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) |
+                        reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(out);
+    if (m % 16 || (qsb | qsn | qsh | ksb | ksn | ksh | osb | osn | osh) % 8) return PYR_ERR_INVALID;
+  }
+  if (c->needs_init) {
+    pyr_status_t st = device_init(c, s);
+    if (st != PYR_OK) return st;
+  }
+  const LayerPlan& p = c->lay.layers[layer];
+  pyr::PrefillArgs a;
+  a.q = q; a.k = k; a.v = v; a.out = out;
+  a.lse = at<float>(c, c->lay.lse);
+  a.score = at<float>(c, c->lay.score);
+  a.w = at<float>(c, c->lay.w) + (c->cfg.recent_len - (p.n_in - p.c));  // newest queries keep their weights
+  a.qsb = qsb; a.qsn = qsn; a.qsh = qsh; a.ksb = ksb; a.ksn = ksn; a.ksh = ksh;
+  a.osb = osb; a.osn = osn; a.osh = osh;
+  a.B = c->cfg.batch; a.n = p.n_in; a.Hq = c->cfg.n_q_heads; a.Hkv = c->cfg.n_kv_heads; a.D = D;
+  a.L = p.n_in - p.c; a.G = c->cfg.sel_groups;
+  a.scale = c->scale; a.dtype = c->cfg.dtype;
+  a.status = at<int>(c, c->lay.status);
+  const bool tc = c->cfg.dtype == PYR_BF16 && !(c->cfg.flags & PYR_FLAG_CUDA_CORE_PREFILL) &&
+                  pyr::prefill_tc_supported(a);
+  cudaError_t e = tc ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
+  if (e != cudaSuccess) return PYR_ERR_CUDA;
+  if (p.c > 0) {
+    e = tc ? pyr::launch_score_tc(a, s) : pyr::launch_score_simt(a, s);
+    if (e != cudaSuccess) return PYR_ERR_CUDA;
+  }
+  c->phase = 1;
+  c->last_prefilled = layer;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, const void* v, int64_t ksb,
+                                int64_t ksn, int64_t ksh, void* rows, int64_t row_elems, int64_t rsb,
+                                int64_t rsn, int64_t rsg, int32_t* n_out, void* stream) {
+  if (!c || !k || !v) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (layer != c->next_layer || c->phase != 1) return PYR_ERR_ORDER;
+  const int D = c->cfg.head_dim;
+  const int eb = c->cfg.dtype == PYR_BF16 ? 2 : 4;
+  if (ksh < D || ksn < D) return PYR_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(k) % 16 || reinterpret_cast<uintptr_t>(v) % 16 ||
+      (ksb * eb) % 16 || (ksn * eb) % 16 || (ksh * eb) % 16)
+    return PYR_ERR_INVALID;
+  if (rows) {
+    if (row_elems < 1 || rsn < row_elems) return PYR_ERR_INVALID;
+    if (c->cfg.sel_groups == 1 ? rsg != 0 : rsg < 1) return PYR_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(rows) % 16 || (row_elems * eb) % 16 || (rsb * eb) % 16 ||
+        (rsn * eb) % 16 || (rsg * eb) % 16)
+      return PYR_ERR_INVALID;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const LayerPlan& p = c->lay.layers[layer];
+  int32_t* pos_in = at<int32_t>(c, c->pos_cur ? c->lay.pos1 : c->lay.pos0);
+  int32_t* pos_out = at<int32_t>(c, c->pos_cur ? c->lay.pos0 : c->lay.pos1);
+
+  pyr::SelectArgs sa;
+  sa.score = at<float>(c, c->lay.score);
+  sa.idx = at<int32_t>(c, c->lay.idx);
+  sa.pos_in = layer == 0 ? nullptr : pos_in;
+  sa.pos_out = pos_out;
+  sa.B = c->cfg.batch; sa.G = c->cfg.sel_groups; sa.n = p.n_in; sa.c = p.c; sa.k = p.k;
+  if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
+
+  pyr::GatherArgs ga;
+  ga.k = k; ga.v = v;
+  ga.kc = c->base + p.k_off; ga.vc = c->base + p.v_off;
+  ga.idx = sa.idx; ga.ksb = ksb; ga.ksn = ksn; ga.ksh = ksh;
+  ga.B = c->cfg.batch; ga.Hkv = c->cfg.n_kv_heads; ga.G = c->cfg.sel_groups; ga.D = D;
+  ga.n_out = p.n_out; ga.cap = p.cap; ga.elem_bytes = eb;
+  if (pyr::launch_gather_kv(ga, s) != cudaSuccess) return PYR_ERR_CUDA;
+
+  if (rows && p.n_out < p.n_in) {
+    pyr::RowsArgs ra;
+    ra.rows = rows; ra.idx = sa.idx; ra.stride_b = rsb; ra.stride_n = rsn; ra.stride_g = rsg;
+    ra.row_elems = row_elems; ra.B = c->cfg.batch; ra.G = c->cfg.sel_groups; ra.n_out = p.n_out;
+    ra.elem_bytes = eb;
+    if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
+  }
+  if (n_out) *n_out = p.n_out;
+  c->len_now[layer] = p.n_out;
+  c->pos_cur ^= 1;
+  c->last_selected = layer;
+  c->next_layer = layer + 1;
+  c->phase = 0;
+  return PYR_OK;
+}
+
+pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                             const void* v_new, void* out, void* stream) {
+  if (!c || !q || !k_new || !v_new || !out) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (c->next_layer != c->cfg.n_layers) return PYR_ERR_ORDER;
+  const LayerPlan& p = c->lay.layers[layer];
+  if (c->len_now[layer] >= p.cap) return PYR_ERR_CAPACITY;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) |
+       reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(out)) % 16)
+    return PYR_ERR_INVALID;
+  pyr::DecodeArgs a;
+  a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out;
+  a.kc = c->base + p.k_off; a.vc = c->base + p.v_off;
+  a.part_acc = at<float>(c, c->lay.part_acc);
+  a.part_ml = at<float>(c, c->lay.part_ml);
+  a.B = c->cfg.batch; a.Hq = c->cfg.n_q_heads; a.Hkv = c->cfg.n_kv_heads; a.D = c->cfg.head_dim;
+  a.len = c->len_now[layer]; a.cap = p.cap;
+  a.scale = c->scale; a.dtype = c->cfg.dtype;
+  // Split the rows so that the grid fills the machine a few times over.
+  const int total = a.len + 1;
+  const long long pairs = (long long)a.B * a.Hkv;
+  int splits = (int)((148LL * 8 + pairs - 1) / pairs);
+  const int max_by_rows = (total + 127) / 128;
+  if (splits > max_by_rows) splits = max_by_rows;
+  if (splits > pyr::kMaxDecodeSplits) splits = pyr::kMaxDecodeSplits;
+  if (splits < 1) splits = 1;
+  int rps = (total + splits - 1) / splits;
+  rps = (rps + 15) / 16 * 16;
+  splits = (total + rps - 1) / rps;
+  a.splits = splits; a.rows_per_split = rps;
+  if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
+  c->len_now[layer] += 1;
+  return PYR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,70 @@
+// Internal declarations shared by the host dispatcher and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pyr.h"
+
+namespace pyr {
+
+constexpr int kStatusWords = 64;
+constexpr int kMaxPrompt = 32768;      // select keeps one sequence's scores in shared memory
+constexpr int kMaxDecodeSplits = 64;
+
+// One layer's attention + score problem.
+struct PrefillArgs {
+  const void* q; const void* k; const void* v; void* out;
+  float* lse;          // [B, Hq, n]
+  float* score;        // [B, G, c] pooled
+  const float* w;      // [L] device
+  int64_t qsb, qsn, qsh, ksb, ksn, ksh, osb, osn, osh;
+  int B, n, Hq, Hkv, D, L, G;   // L = window actually present (min(L, n)); c = n - L
+  float scale;
+  int dtype;
+  int* status;
+};
+
+struct SelectArgs {
+  const float* score;  // [B, G, c]
+  int32_t* idx;        // [B, G, n_out]
+  const int32_t* pos_in;   // [B, G, n] or nullptr = identity
+  int32_t* pos_out;    // [B, G, n_out]
+  int B, G, n, c, k;   // n_out = k + (n - c)
+};
+
+struct GatherArgs {
+  const void* k; const void* v;    // [B, n, Hkv, D] strided
+  void* kc; void* vc;              // [B, Hkv, cap, D]
+  const int32_t* idx;              // [B, G, n_out]
+  int64_t ksb, ksn, ksh;
+  int B, Hkv, G, D, n_out, cap, elem_bytes;
+};
+
+struct RowsArgs {
+  void* rows; const int32_t* idx;
+  int64_t stride_b, stride_n, stride_g;   // elements
+  int64_t row_elems;
+  int B, G, n_out, elem_bytes;
+};
+
+struct DecodeArgs {
+  const void* q; const void* k_new; const void* v_new; void* out;
+  void* kc; void* vc;              // [B, Hkv, cap, D]
+  float* part_acc;                 // [B, Hq, splits, D]
+  float* part_ml;                  // [B, Hq, splits, 2]
+  int B, Hq, Hkv, D, len, cap, splits, rows_per_split;   // len = rows before the append
+  float scale;
+  int dtype;
+};
+
+cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t s);
+cudaError_t launch_score_simt(const PrefillArgs& a, cudaStream_t s);
+cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s);     // bf16, D = 128, tcgen05
+cudaError_t launch_score_tc(const PrefillArgs& a, cudaStream_t s);
+bool prefill_tc_supported(const PrefillArgs& a);
+cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);
+cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s);
+cudaError_t launch_compact_rows(const RowsArgs& a, cudaStream_t s);
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s);
+
+}  // namespace pyr

@@ -1,0 +1,143 @@
+"""Host side of the C ABI, no GPU: the library loads, exports what the header
+declares, validates arguments, orders calls, and turns the ratio schedule into
+the same integer budgets as the oracle."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import oracle
+from paper_2405_12532_b200 import binding as pb
+from paper_2405_12532_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+FAKE_DEV = 0x7F0000000000          # never dereferenced on the host
+
+
+def _cfg(**over):
+    kw = dict(n_layers=4, n_q_heads=8, n_kv_heads=4, head_dim=128, sel_groups=4, dtype="bf16", batch=2,
+              prompt_len=512, recent_len=64, max_new_tokens=8, ratio=[1.0, 0.8, 0.5, 0.5])
+    kw.update(over)
+    return pb.make_config(**kw)
+
+
+def _alloc(**over):
+    cfg, keep = _cfg(**over)
+    nbytes, align = pb.pyr_cache_bytes(cfg)
+    h = C.c_void_p()
+    st = pb.lib().pyr_cache_alloc(C.byref(cfg), C.c_void_p(FAKE_DEV), nbytes, C.byref(h))
+    assert st == pb.PYR_OK
+    return h, cfg, keep, nbytes
+
+
+def test_library_exports_every_declared_symbol():
+    with open(os.path.join(ROOT, "include", "pyr.h")) as f:
+        text = f.read()
+    declared = set(re.findall(r"\b(pyr_[a-z_]+)\s*\(", text))
+    assert declared == set(pb.EXPORTS)
+    L = pb.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert L.pyr_version() >= 100
+    assert pb.status_string(pb.PYR_ERR_ORDER) == "call out of sequence"
+
+
+@pytest.mark.parametrize("over,want", [
+    (dict(n_q_heads=6, n_kv_heads=4), pb.PYR_ERR_INVALID),
+    (dict(sel_groups=2), pb.PYR_ERR_INVALID),
+    (dict(head_dim=96), pb.PYR_ERR_UNSUPPORTED),
+    (dict(dtype=7), pb.PYR_ERR_UNSUPPORTED),
+    (dict(ratio=[1.0, 0.8, 0.9, 0.5]), pb.PYR_ERR_INVALID),      # increasing
+    (dict(ratio=[1.2, 0.8, 0.5, 0.5]), pb.PYR_ERR_INVALID),
+    (dict(ratio=[1.0, 0.8, 0.5, -0.1]), pb.PYR_ERR_INVALID),
+    (dict(recent_len=0), pb.PYR_ERR_INVALID),
+    (dict(batch=0), pb.PYR_ERR_INVALID),
+    (dict(prompt_len=1 << 20), pb.PYR_ERR_UNSUPPORTED),
+    (dict(recent_w=[-1.0] * 64), pb.PYR_ERR_INVALID),
+    (dict(softmax_scale=-1.0), pb.PYR_ERR_INVALID),
+    (dict(min_len=[0, 0, -3, 0]), pb.PYR_ERR_INVALID),
+    (dict(ratio=None), pb.PYR_ERR_NULL),
+])
+def test_config_validation(over, want):
+    cfg, keep = _cfg(**over)
+    b = C.c_size_t(0)
+    assert pb.lib().pyr_cache_bytes(C.byref(cfg), C.byref(b), None) == want
+
+
+def test_null_and_small_buffer():
+    L = pb.lib()
+    cfg, keep = _cfg()
+    b = C.c_size_t(0)
+    assert L.pyr_cache_bytes(None, C.byref(b), None) == pb.PYR_ERR_NULL
+    assert L.pyr_cache_bytes(C.byref(cfg), None, None) == pb.PYR_ERR_NULL
+    nbytes, align = pb.pyr_cache_bytes(cfg)
+    assert align == 256
+    h = C.c_void_p()
+    assert L.pyr_cache_alloc(C.byref(cfg), None, nbytes, C.byref(h)) == pb.PYR_ERR_NULL
+    assert L.pyr_cache_alloc(C.byref(cfg), C.c_void_p(FAKE_DEV), nbytes - 1, C.byref(h)) == pb.PYR_ERR_BUFFER_TOO_SMALL
+    assert L.pyr_cache_alloc(C.byref(cfg), C.c_void_p(FAKE_DEV + 8), nbytes, C.byref(h)) == pb.PYR_ERR_INVALID
+    assert L.pyr_cache_free(None) == pb.PYR_ERR_NULL
+
+
+def _info(h, layer):
+    v = [C.c_int32(0) for _ in range(4)]
+    st = pb.lib().pyr_cache_layer_info(h, layer, *[C.byref(x) for x in v])
+    return st, [x.value for x in v]
+
+
+@pytest.mark.parametrize("name", list(synth.CONFIGS))
+def test_budgets_equal_oracle_on_all_workloads(name):
+    w = synth.CONFIGS[name]
+    ratio = synth.ratio_schedule(w)
+    h, cfg, keep, nbytes = _alloc(**pb.config_from_workload(w, ratio))
+    want = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
+    for l, b in enumerate(want):
+        st, (n_in, k, len_now, cap) = _info(h, l)
+        assert st == pb.PYR_OK
+        assert (n_in, k, len_now, cap) == (b["n_in"], b["k"], 0, b["n_out"] + w["max_new_tokens"])
+    eb = 2 if w["dtype"] == "bf16" else 4
+    kv = oracle.cache_bytes(w["batch"], w["n_kv_heads"], w["head_dim"], eb, w["prompt_len"], w["recent_len"],
+                            ratio, w["max_new_tokens"])
+    assert kv <= nbytes <= kv * 1.08 + (64 << 20)
+    assert _info(h, w["n_layers"])[0] == pb.PYR_ERR_INVALID
+    pb.lib().pyr_cache_free(h)
+
+
+def test_budget_edges_match_oracle():
+    for N, L, ratio, ml in [(20, 32, [0.5, 0.1], None), (100, 10, [0.0], None),
+                            (100, 10, [0.1, 0.1], [50, 60]), (100, 10, [0.9, 0.5], None),
+                            (4097, 1, [1.0, 0.33333, 0.001], None)]:
+        h, cfg, keep, _ = _alloc(n_layers=len(ratio), prompt_len=N, recent_len=L, ratio=ratio, min_len=ml)
+        for l, b in enumerate(oracle.layer_budgets(N, L, ratio, ml)):
+            st, (n_in, k, _, cap) = _info(h, l)
+            assert (n_in, k, cap) == (b["n_in"], b["k"], b["n_out"] + 8)
+        pb.lib().pyr_cache_free(h)
+
+
+def test_call_order_and_pointer_checks_before_any_launch():
+    L = pb.lib()
+    h, cfg, keep, _ = _alloc()
+    p = C.c_void_p(FAKE_DEV)
+    st = [64 * 8 * 128, 8 * 128, 128, 64 * 4 * 128, 4 * 128, 128, 64 * 8 * 128, 8 * 128, 128]
+    # wrong layer, select before prefill, decode before the prompt is done
+    assert L.pyr_prefill_layer(h, 1, p, p, p, p, *st, None) == pb.PYR_ERR_ORDER
+    assert L.pyr_select_compact(h, 0, p, p, st[3], st[4], st[5], None, 0, 0, 0, 0, None, None) == pb.PYR_ERR_ORDER
+    assert L.pyr_decode_attn(h, 0, p, p, p, p, None) == pb.PYR_ERR_ORDER
+    assert L.pyr_prefill_layer(h, 0, None, p, p, p, *st, None) == pb.PYR_ERR_NULL
+    assert L.pyr_prefill_layer(h, 9, p, p, p, p, *st, None) == pb.PYR_ERR_INVALID
+    bad = list(st); bad[2] = 64                      # head stride smaller than D
+    assert L.pyr_prefill_layer(h, 0, p, p, p, p, *bad, None) == pb.PYR_ERR_INVALID
+    bad = list(st); bad[1] = 8 * 128 + 3             # bf16 rows must stay 16-byte aligned
+    assert L.pyr_prefill_layer(h, 0, p, p, p, p, *bad, None) == pb.PYR_ERR_INVALID
+    ip, pp = C.c_void_p(), C.c_void_p()
+    assert L.pyr_cache_kept(h, 0, C.byref(ip), C.byref(pp)) == pb.PYR_ERR_ORDER
+    assert L.pyr_cache_scores(h, 0, C.byref(ip)) == pb.PYR_ERR_ORDER
+    L.pyr_cache_free(h)
+
+
+def test_shard_batch_covers_batch():
+    for B, W in [(64, 8), (10, 4), (3, 4)]:
+        spans = [synth.shard_batch(B, W, r) for r in range(W)]
+        assert spans[0][0] == 0 and spans[-1][1] == B
+        assert all(spans[i][1] == spans[i + 1][0] for i in range(W - 1))

@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the pyramid prefill-selection path.
+
+One step = one pass of the whole path over one synthetic batch: for every layer
+attention + recent-window score, then top-k + K/V gather + in-place compaction
+of the hidden rows; then T decode steps over the ragged per-layer caches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line. Under torchrun every rank runs the same per-GPU workload
+(sequences are independent: weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2405_12532_b200 import synth
+
+METRIC = "prefill tokens/s + decode tokens/s at 7B shapes 64x2k"
+DEFAULT_WORKLOAD = "7b_64x2k"
+
+
+def measured_peaks():
+    """(hbm GB/s, bf16 TFLOP/s burst, source)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p["bf16_tflops"]), float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "measured"
+    return 6650.0, 1590.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ ours
+class Workload:
+    """Device-resident synthetic inputs and the call sequence of one step."""
+
+    def __init__(self, name: str, device, pool: int = 2):
+        from paper_2405_12532_b200 import binding as pb
+        self.pb = pb
+        self.name = name
+        self.w = w = synth.CONFIGS[name]
+        self.device = device
+        self.ratio = synth.ratio_schedule(w)
+        self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio))
+        self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
+        B, N, Hq, Hkv, D = w["batch"], w["prompt_len"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
+        self.dt = synth.torch_dtype(w["dtype"])
+        self.eb = 2 if w["dtype"] == "bf16" else 4
+        # a small pool of full-length Q/K/V sets; layer l reads the first n_in rows of set l % pool
+        # (values do not change the work done; every tensor is far larger than L2)
+        self.pool = [synth.stack_layer_inputs(w, l, N, device=device) for l in range(pool)]
+        self.out = torch.empty(B, N, Hq, D, dtype=self.dt, device=device)
+        self.G = w["sel_groups"]
+        if self.G == 1:
+            self.hidden = w.get("hidden", Hq * D)
+            self.rows = torch.randn(B, N, self.hidden, device=device).to(self.dt)
+        else:
+            self.rows = None
+        self.T = w["max_new_tokens"]
+        self.dec_in = [synth.decode_step_inputs(w, 0, t, device=device) for t in range(4)]
+        self.dec_out = torch.empty(B, Hq, D, dtype=self.dt, device=device)
+
+    def layer_views(self, l):
+        n = self.layers[l]["n_in"]
+        Q, K, V = self.pool[l % len(self.pool)]
+        return Q[:, :n], K[:, :n], V[:, :n], self.out[:, :n], n
+
+    def select_args(self, l, n):
+        w = self.w
+        if self.G == 1:
+            return (self.rows, self.hidden, self.rows.stride(0), self.hidden, 0)
+        rep = w["n_q_heads"] // w["n_kv_heads"]
+        D = w["head_dim"]
+        return (self.out, rep * D, self.out.stride(0), self.out.stride(1), rep * D)
+
+    def prefill(self, events=None):
+        c = self.cache
+        c.reset()
+        for l in range(self.w["n_layers"]):
+            Q, K, V, O, n = self.layer_views(l)
+            if events is not None:
+                events[l][0].record()
+            c.prefill_layer(l, Q, K, V, O)
+            if events is not None:
+                events[l][1].record()
+            c.select_compact(l, K, V, *self.select_args(l, n))
+            if events is not None:
+                events[l][2].record()
+
+    def decode(self):
+        c = self.cache
+        for t in range(self.T):
+            q, kn, vn = self.dec_in[t % len(self.dec_in)]
+            for l in range(self.w["n_layers"]):
+                c.decode_attn(l, q, kn, vn, self.dec_out)
+
+    # ---- algorithmic work, from the schedule
+    def prefill_flops(self):
+        w = self.w
+        return sum(w["batch"] * w["n_q_heads"] * 2 * w["head_dim"] * L["n_in"] * (L["n_in"] + 1) for L in self.layers)
+
+    def select_compact_bytes(self):
+        w = self.w
+        B, Hkv, D, G, Lw = w["batch"], w["n_kv_heads"], w["head_dim"], self.G, w["recent_len"]
+        tot = 0
+        for L in self.layers:
+            n = L["n_in"]
+            c = max(n - Lw, 0)
+            n_out = L["k_ctx"] + (n - c)
+            tot += B * G * c * 4 + B * G * n_out * 4                        # scores in, indices out
+            tot += 2 * 2 * B * Hkv * n_out * D * self.eb                    # K and V, read + write
+            if n_out < n:
+                row_b = (self.hidden if G == 1 else (w["n_q_heads"] // Hkv) * D) * self.eb
+                tot += 2 * B * G * n_out * row_b                            # compacted rows, read + write
+            tot += 2 * B * G * n_out * 4                                    # positions
+        return tot
+
+    def decode_bytes(self):
+        w = self.w
+        tot = 0
+        for L in self.layers:
+            n_out = L["k_ctx"] + min(w["recent_len"], L["n_in"])
+            for t in range(self.T):
+                tot += 2 * w["batch"] * w["n_kv_heads"] * (n_out + t + 1) * w["head_dim"] * self.eb
+        return tot
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2405_12532_b200 import binding as pb
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    wl = Workload(args.workload, device)
+    w = wl.w
+    nL = w["n_layers"]
+    hbm, tf_burst, tf_sust, peak_src = measured_peaks()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        wl.prefill(); wl.decode()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = pb.launch_count()
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(nL)] for _ in range(args.steps)]
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        marks[s][0].record()
+        wl.prefill(ev[s])
+        marks[s][1].record()
+        wl.decode()
+        marks[s][2].record()
+    barrier()
+    wall = time.perf_counter() - t0
+    launches = pb.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    assert wl.cache.status() == 0, "device-side wait timed out"
+
+    t_pre = sum(m[0].elapsed_time(m[1]) for m in marks) / 1e3
+    t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
+    t_attn = sum(e[0].elapsed_time(e[1]) for st in ev for e in st) / 1e3
+    t_sel = sum(e[1].elapsed_time(e[2]) for st in ev for e in st) / 1e3
+    times = torch.tensor([t_pre, t_dec, t_attn, t_sel, t_pre + t_dec], dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
+    t_pre, t_dec, t_attn, t_sel, t_all = [float(x) for x in times.tolist()]
+
+    K = args.steps
+    B, N, T = w["batch"], w["prompt_len"], w["max_new_tokens"]
+    prefill_tps = world * K * B * N / t_pre
+    decode_tps = world * K * B * T / t_dec if T > 0 and t_dec > 0 else None
+
+    # ---- end to end: host buffers, copies inside the timed region
+    e2e = run_e2e(wl, args, barrier, world) if not args.no_e2e else None
+
+    if rank != 0:
+        return
+    dec_bytes = wl.decode_bytes()
+    dec_launches = nL * T
+    roof_dec = None
+    if T > 0:
+        ach = K * dec_bytes / t_dec / 1e9
+        roof_dec = {"kernel": "decode_kernel", "bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s",
+                    "frac": ach / hbm, "traffic": None, "peak_source": f"of {peak_src}",
+                    "launches": K * dec_launches, "avg_launch_us": t_dec / (K * dec_launches) * 1e6,
+                    "algorithmic_bytes_per_launch": dec_bytes / dec_launches}
+    ach_tf = K * wl.prefill_flops() / t_attn / 1e12
+    roof_pre = {"kernel": "prefill attention + score", "bound": "tensor", "achieved": ach_tf, "peak": tf_burst,
+                "unit": "TFLOP/s", "frac": ach_tf / tf_burst, "frac_of_sustained": ach_tf / tf_sust,
+                "traffic": None, "peak_source": f"of {peak_src}", "launches": K * nL * 2,
+                "avg_layer_us": t_attn / (K * nL) * 1e6}
+    ach_sel = K * wl.select_compact_bytes() / t_sel / 1e9
+    roof_sel = {"kernel": "select + gather + compact", "bound": "hbm", "achieved": ach_sel, "peak": hbm,
+                "unit": "GB/s", "frac": ach_sel / hbm, "traffic": None, "peak_source": f"of {peak_src}",
+                "avg_layer_us": t_sel / (K * nL) * 1e6}
+    dominant = roof_dec if (roof_dec and t_dec >= t_attn) else roof_pre
+    line = {
+        "metric": METRIC, "value": prefill_tps, "unit": "tokens/s (prefill, all layers incl. select+compact)",
+        "decode_tokens_per_s": decode_tps,
+        "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": t_all / K * 1e3,
+        "ms_prefill": t_pre / K * 1e3, "ms_decode": t_dec / K * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "layers": nL, "batch_per_gpu": B, "prompt_len": N,
+                   "recent_len": w["recent_len"], "decode_steps": T, "sel_groups": w["sel_groups"],
+                   "heads": w["n_q_heads"], "kv_heads": w["n_kv_heads"], "head_dim": w["head_dim"],
+                   "ratio": "geometric 1.0->%.2f" % wl.ratio[-1],
+                   "l2": "inputs larger than L2 (each of Q, K, V and the cache is >= 1 GB)"},
+        "roofline": dominant, "roofline_prefill": roof_pre, "roofline_select_compact": roof_sel,
+        "roofline_decode": roof_dec,
+        "gpu_launches": launches, "wall_s": wall, "clocks": clocks, "e2e": e2e,
+        "cpu_baseline": cpu_baseline(args.workload) if not args.no_cpu else None,
+    }
+    print(json.dumps(line))
+
+
+def run_e2e(wl, args, barrier, world):
+    """The same step driven from pinned host buffers: each layer's Q/K/V are
+    copied host->device before its calls, the last layer's attention output and
+    every decode output are copied back."""
+    w = wl.w
+    steps = max(1, min(args.steps, args.e2e_steps))
+    host_pool = [tuple(x.to("cpu").pin_memory() for x in qkv) for qkv in wl.pool[:1]]
+    hq, hk, hv = host_pool[0]
+    dq, dk, dv = wl.pool[0]
+    dec_host = [tuple(x.to("cpu").pin_memory() for x in d) for d in wl.dec_in[:1]]
+    out_host = torch.empty(wl.out.shape, dtype=wl.out.dtype).pin_memory()
+    dec_out_host = torch.empty(wl.dec_out.shape, dtype=wl.dec_out.dtype).pin_memory()
+    c = wl.cache
+    nL = w["n_layers"]
+    h2d = d2h = 0
+
+    def step(count):
+        nonlocal h2d, d2h
+        c.reset()
+        for l in range(nL):
+            n = wl.layers[l]["n_in"]
+            for src, dst in ((hq, dq), (hk, dk), (hv, dv)):
+                dst[:, :n].copy_(src[:, :n], non_blocking=True)
+                if count:
+                    h2d += src[:, :n].numel() * src.element_size()
+            O = wl.out[:, :n]
+            c.prefill_layer(l, dq[:, :n], dk[:, :n], dv[:, :n], O)
+            c.select_compact(l, dk[:, :n], dv[:, :n], *wl.select_args(l, n))
+        n_last = wl.layers[-1]["n_in"]
+        out_host[:, :n_last].copy_(wl.out[:, :n_last], non_blocking=True)
+        if count:
+            d2h += wl.out[:, :n_last].numel() * wl.out.element_size()
+        q, kn, vn = wl.dec_in[0]
+        hq1, hk1, hv1 = dec_host[0]
+        for t in range(wl.T):
+            for l in range(nL):
+                q.copy_(hq1, non_blocking=True); kn.copy_(hk1, non_blocking=True); vn.copy_(hv1, non_blocking=True)
+                c.decode_attn(l, q, kn, vn, wl.dec_out)
+                dec_out_host.copy_(wl.dec_out, non_blocking=True)
+                if count:
+                    h2d += (q.numel() + kn.numel() + vn.numel()) * q.element_size()
+                    d2h += wl.dec_out.numel() * wl.dec_out.element_size()
+
+    step(False)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step(True)
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1) / 1e3], dtype=torch.float64, device=wl.device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    t = float(t.item())
+    B, N, T = w["batch"], w["prompt_len"], w["max_new_tokens"]
+    return {"value": world * steps * B * (N + T) / t, "unit": "tokens/s (prompt + generated, whole step from host buffers)",
+            "steps": steps, "ms_per_step": t / steps * 1e3,
+            "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps}
+
+
+# ------------------------------------------------------------------------------------------ oracle
+def oracle_sample(workload: str, layers=None):
+    """Times the fp64 oracle, as it stands, on ONE sequence of the workload at a
+    few layers; returns (seconds, description, est. prefill tokens/s for a full pass)."""
+    import numpy as np
+    import oracle
+    w = synth.CONFIGS[workload]
+    ratio = synth.ratio_schedule(w)
+    budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
+    nL = len(budgets)
+    layers = layers or sorted({0, nL // 2, nL - 1})
+    cores = len(os.sched_getaffinity(0))
+    torch.set_num_threads(cores)
+    t_total = 0.0
+    for l in layers:
+        bud = budgets[l]
+        Q, K, V = synth.stack_layer_inputs(w, l, bud["n_in"], device="cpu", batch=1)
+        Qn, Kn, Vn = synth.widen(Q), synth.widen(K), synth.widen(V)
+        t0 = time.perf_counter()
+        oracle.prefill_layer(Qn, Kn, Vn, w["recent_len"], bud["k"], w["sel_groups"])
+        t_total += time.perf_counter() - t0
+    work = lambda ls: sum(budgets[l]["n_in"] ** 2 for l in ls)
+    t_full = t_total * work(range(nL)) / work(layers)
+    desc = (f"1 of {w['batch']} sequences, layers {layers} of {nL} (attention + score + top-k + gather), "
+            f"scaled to all layers by sum of n_in^2")
+    return t_total, desc, w["prompt_len"] / t_full, cores
+
+
+def cpu_baseline(workload: str):
+    t, desc, tps, cores = oracle_sample(workload)
+    return {"value": tps, "unit": "tokens/s (prefill, estimated from the sample)", "cores": cores, "kind": "oracle",
+            "sample": desc, "sample_seconds": t}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    w = synth.CONFIGS[args.workload]
+    nL = w["n_layers"]
+    per_step = []
+    desc = cores = None
+    for i in range(args.warmup + args.steps):
+        layers = [0] if i < args.warmup else [nL - 1]      # warm-up: one layer; timed: the smallest layer
+        t0 = time.perf_counter()
+        t, desc, tps, cores = oracle_sample(args.workload, layers)
+        if i >= args.warmup:
+            per_step.append((time.perf_counter() - t0, tps))
+    value = statistics.mean(x[1] for x in per_step)
+    ms = statistics.mean(x[0] for x in per_step) * 1e3
+    unit = "tokens/s (prefill, estimated from the sample)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(synth.CONFIGS))
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -203,6 +203,9 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, c
 
 const char* pyr_status_string(pyr_status_t status);
 
+/* Number of kernels this process has launched through the library so far. */
+uint64_t pyr_launch_count(void);
+
 /* Library version: major*10000 + minor*100 + patch. */
 int32_t pyr_version(void);
 

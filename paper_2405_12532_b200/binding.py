@@ -21,7 +21,7 @@ PYR_FLAG_CUDA_CORE_PREFILL = 1
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_status_string", "pyr_version",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_status_string", "pyr_version", "pyr_launch_count",
 ]
 
 
@@ -59,6 +59,8 @@ def lib() -> C.CDLL:
         L.pyr_status_string.restype = C.c_char_p
         L.pyr_status_string.argtypes = [C.c_int]
         L.pyr_version.restype = i32
+        L.pyr_launch_count.restype = C.c_uint64
+        L.pyr_launch_count.argtypes = []
         L.pyr_cache_bytes.argtypes = [C.POINTER(PyrConfig), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
         L.pyr_cache_alloc.argtypes = [C.POINTER(PyrConfig), vp, C.c_size_t, C.POINTER(vp)]
         L.pyr_cache_free.argtypes = [vp]
@@ -74,10 +76,14 @@ def lib() -> C.CDLL:
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             fn = getattr(L, name)
-            if name not in ("pyr_status_string", "pyr_version"):
+            if name not in ("pyr_status_string", "pyr_version", "pyr_launch_count"):
                 fn.restype = C.c_int
         _lib = L
     return _lib
+
+
+def launch_count() -> int:
+    return int(lib().pyr_launch_count())
 
 
 def status_string(status: int) -> str:

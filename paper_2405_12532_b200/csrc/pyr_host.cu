@@ -2,6 +2,7 @@
 // (Algorithm 1: ratio p per layer, minimum PvC lengths N_l), carving of the
 // caller's device buffer, call ordering, and dispatch to the kernels.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -19,6 +20,8 @@ struct LayerPlan {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 constexpr size_t kAlign = 256;
+
+std::atomic<uint64_t> g_launches{0};   // kernels launched by this process through the library
 
 struct Layout {
   size_t status, w, score, lse, idx, pos0, pos1, part_acc, part_ml, total;
@@ -157,6 +160,8 @@ const char* pyr_status_string(pyr_status_t s) {
 }
 
 int32_t pyr_version(void) { return 100; }
+
+uint64_t pyr_launch_count(void) { return g_launches.load(); }
 
 pyr_status_t pyr_cache_bytes(const pyr_config_t* cfg, size_t* bytes, size_t* align) {
   pyr_status_t st = validate(cfg);
@@ -302,9 +307,11 @@ pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, con
                   pyr::prefill_tc_supported(a);
   cudaError_t e = tc ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
   if (e != cudaSuccess) return PYR_ERR_CUDA;
+  g_launches += 1;
   if (p.c > 0) {
     e = tc ? pyr::launch_score_tc(a, s) : pyr::launch_score_simt(a, s);
     if (e != cudaSuccess) return PYR_ERR_CUDA;
+    g_launches += 1;
   }
   c->phase = 1;
   c->last_prefilled = layer;
@@ -350,6 +357,7 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
   ga.B = c->cfg.batch; ga.Hkv = c->cfg.n_kv_heads; ga.G = c->cfg.sel_groups; ga.D = D;
   ga.n_out = p.n_out; ga.cap = p.cap; ga.elem_bytes = eb;
   if (pyr::launch_gather_kv(ga, s) != cudaSuccess) return PYR_ERR_CUDA;
+  g_launches += 2;
 
   if (rows && p.n_out < p.n_in) {
     pyr::RowsArgs ra;
@@ -357,6 +365,7 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
     ra.row_elems = row_elems; ra.B = c->cfg.batch; ra.G = c->cfg.sel_groups; ra.n_out = p.n_out;
     ra.elem_bytes = eb;
     if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
+    g_launches += 1;
   }
   if (n_out) *n_out = p.n_out;
   c->len_now[layer] = p.n_out;
@@ -398,6 +407,7 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   splits = (total + rps - 1) / rps;
   a.splits = splits; a.rows_per_split = rps;
   if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
+  g_launches += splits > 1 ? 2 : 1;
   c->len_now[layer] += 1;
   return PYR_OK;
 }

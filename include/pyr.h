@@ -62,7 +62,8 @@ typedef enum {
   PYR_ERR_CAPACITY = 5,         /* decode append beyond max_new_tokens             */
   PYR_ERR_ORDER = 6,            /* call out of the prefill/select/decode sequence  */
   PYR_ERR_CUDA = 7,             /* a CUDA runtime call failed                      */
-  PYR_ERR_TIMEOUT = 8           /* a bounded device-side wait ran out              */
+  PYR_ERR_TIMEOUT = 8,          /* a bounded device-side wait ran out              */
+  PYR_ERR_SCRATCH_LIMIT = 9     /* problem exceeds the library's built-in scratch  */
 } pyr_status_t;
 
 typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
@@ -200,6 +201,43 @@ pyr_status_t pyr_select_compact(pyr_cache_t* cache, int32_t layer, const void* k
  */
 pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, const void* k_new,
                              const void* v_new, void* out, void* stream);
+
+/*
+ * Decode attention for callers that must not allocate device memory.
+ * (No counterpart in the paper: this is a packaging variant of pyr_decode_attn.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they
+ * decode: code running inside a serving engine that has handed all device
+ * memory to its own pool, plugins that are only given tensors, code on a
+ * latency path where an allocation (an implicit device synchronisation) is not
+ * acceptable. pyr_decode_attn needs a cache handle whose buffer includes a
+ * split-K workspace; this entry point needs neither. The caller passes only
+ * inputs and outputs:
+ *   q [B, Hq, D], k_new / v_new [B, Hkv, D], out [B, Hq, D]      (device, contiguous)
+ *   k_cache / v_cache [B, Hkv, cap, D] with rows 0..len-1 filled (device)
+ * The new row is stored at row `len` of both caches and q attends over rows
+ * 0..len, exactly as pyr_decode_attn does; the caller advances `len` itself.
+ * softmax_scale 0 means 1/sqrt(D).
+ *
+ * The split-K partial results go to an array compiled into the library
+ * (4 MiB per GPU, resident on every GPU that loads the library until the
+ * process exits). A call whose B * Hq * splits * (D + 2) floats exceed it
+ * returns PYR_ERR_SCRATCH_LIMIT and launches nothing; the split count is
+ * min(64, ceil(1184 / (B * Hkv)), ceil((len + 1) / 128)) before rounding the
+ * rows per split up to 16, and with one split no scratch is used at all.
+ * All calls on a GPU share that array and it keeps the previous call's
+ * contents (every slot is rewritten before it is read, so none needs
+ * clearing): two calls whose kernels can overlap on the GPU - different
+ * streams, or different threads - race on it; keep them on one stream or
+ * order them with events. The first call on each GPU looks the array's device
+ * address up, which is a CUDA runtime call outside the stream: make that
+ * first call before any stream capture begins. No cudaMalloc, cudaFree or
+ * other allocating routine is called, on any call.
+ */
+pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new, const void* v_new, void* out,
+                                     void* k_cache, void* v_cache, int32_t batch, int32_t n_q_heads,
+                                     int32_t n_kv_heads, int32_t head_dim, int32_t dtype, int32_t len,
+                                     int32_t cap, float softmax_scale, void* stream);
 
 const char* pyr_status_string(pyr_status_t status);
 

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libpyr.so")
 
 PYR_OK, PYR_ERR_INVALID, PYR_ERR_NULL, PYR_ERR_UNSUPPORTED, PYR_ERR_BUFFER_TOO_SMALL, \
     PYR_ERR_CAPACITY, PYR_ERR_ORDER, PYR_ERR_CUDA, PYR_ERR_TIMEOUT = range(9)
+PYR_ERR_SCRATCH_LIMIT = 9
 PYR_BF16, PYR_F32 = 0, 1
 PYR_FLAG_CUDA_CORE_PREFILL = 1
 
@@ -22,6 +23,7 @@ EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
     "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_status_string", "pyr_version", "pyr_launch_count",
+    "pyr_decode_attn_noalloc",
 ]
 
 
@@ -74,6 +76,8 @@ def lib() -> C.CDLL:
         L.pyr_prefill_layer.argtypes = [vp, i32, vp, vp, vp, vp] + [i64] * 9 + [vp]
         L.pyr_select_compact.argtypes = [vp, i32, vp, vp, i64, i64, i64, vp, i64, i64, i64, i64, pi32, vp]
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+        L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                              C.c_float, vp]
         for name in EXPORTS:
             fn = getattr(L, name)
             if name not in ("pyr_status_string", "pyr_version", "pyr_launch_count"):
@@ -132,6 +136,19 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return int(stream.cuda_stream)
+
+
+def decode_attn_noalloc(q, k_new, v_new, out, k_cache, v_cache, length: int, softmax_scale: float = 0.0,
+                        stream=None) -> int:
+    """pyr_decode_attn_noalloc on torch tensors (q [B,Hq,D], k_new/v_new [B,Hkv,D],
+    caches [B,Hkv,cap,D], `length` rows filled). Returns the status code; the
+    library allocates nothing and the binding only reads pointers and shapes."""
+    B, Hq, D = q.shape
+    Hkv, cap = k_cache.shape[1], k_cache.shape[2]
+    dt = PYR_BF16 if q.dtype == torch.bfloat16 else PYR_F32
+    return lib().pyr_decode_attn_noalloc(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+                                         k_cache.data_ptr(), v_cache.data_ptr(), B, Hq, Hkv, D, dt, int(length),
+                                         cap, float(softmax_scale), C.c_void_p(_stream_ptr(stream)))
 
 
 def config_from_workload(w: dict, ratio, **over) -> dict:

@@ -155,6 +155,7 @@ const char* pyr_status_string(pyr_status_t s) {
     case PYR_ERR_ORDER: return "call out of sequence";
     case PYR_ERR_CUDA: return "CUDA runtime error";
     case PYR_ERR_TIMEOUT: return "device-side wait timed out";
+    case PYR_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in array holds";
   }
   return "unknown status";
 }

@@ -304,13 +304,14 @@ pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, con
   a.L = p.n_in - p.c; a.G = c->cfg.sel_groups;
   a.scale = c->scale; a.dtype = c->cfg.dtype;
   a.status = at<int>(c, c->lay.status);
-  const bool tc = c->cfg.dtype == PYR_BF16 && !(c->cfg.flags & PYR_FLAG_CUDA_CORE_PREFILL) &&
-                  pyr::prefill_tc_supported(a);
-  cudaError_t e = tc ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
+  const bool want_tc = c->cfg.dtype == PYR_BF16 && !(c->cfg.flags & PYR_FLAG_CUDA_CORE_PREFILL);
+  const bool tc_attn = want_tc && pyr::prefill_tc_supported(a);
+  const bool tc_score = want_tc && pyr::score_tc_supported(a);
+  cudaError_t e = tc_attn ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
   if (e != cudaSuccess) return PYR_ERR_CUDA;
   g_launches += 1;
   if (p.c > 0) {
-    e = tc ? pyr::launch_score_tc(a, s) : pyr::launch_score_simt(a, s);
+    e = tc_score ? pyr::launch_score_tc(a, s) : pyr::launch_score_simt(a, s);
     if (e != cudaSuccess) return PYR_ERR_CUDA;
     g_launches += 1;
   }

@@ -62,6 +62,7 @@ cudaError_t launch_score_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s);     // bf16, D = 128, tcgen05
 cudaError_t launch_score_tc(const PrefillArgs& a, cudaStream_t s);
 bool prefill_tc_supported(const PrefillArgs& a);
+bool score_tc_supported(const PrefillArgs& a);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s);
 cudaError_t launch_compact_rows(const RowsArgs& a, cudaStream_t s);

@@ -123,6 +123,8 @@ SHAPES = [
     ("bf16", 2, 2, 2, 128, 1, 130, 30, 0),         # k = 0: only the window survives
     ("bf16", 2, 2, 2, 128, 1, 130, 30, 100),       # k = c: keep everything
     ("bf16", 2, 1, 1, 128, 1, 1, 1, 0),            # a single token
+    ("bf16", 2, 2, 2, 128, 1, 1100, 200, 333),     # several key tiles per query tile, ragged last pair
+    ("bf16", 4, 1, 1, 128, 2, 1536, 256, 700),     # GQA, six full query-tile pairs
 ]
 
 

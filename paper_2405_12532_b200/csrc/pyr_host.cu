@@ -396,6 +396,7 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   a.B = c->cfg.batch; a.Hq = c->cfg.n_q_heads; a.Hkv = c->cfg.n_kv_heads; a.D = c->cfg.head_dim;
   a.len = c->len_now[layer]; a.cap = p.cap;
   a.scale = c->scale; a.dtype = c->cfg.dtype;
+  a.status = at<int>(c, c->lay.status);
   // Split the rows so that the grid fills the machine a few times over.
   const int total = a.len + 1;
   const long long pairs = (long long)a.B * a.Hkv;

@@ -55,6 +55,7 @@ struct DecodeArgs {
   int B, Hq, Hkv, D, len, cap, splits, rows_per_split;   // len = rows before the append
   float scale;
   int dtype;
+  int* status;                     // device status word, may be null
 };
 
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t s);

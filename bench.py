@@ -98,13 +98,18 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs and the call sequence of one step."""
 
-    def __init__(self, name: str, device, pool: int = 2):
+    def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1):
         from paper_2405_12532_b200 import binding as pb
         self.pb = pb
         self.name = name
-        self.w = w = synth.CONFIGS[name]
+        self.w = w = dict(synth.CONFIGS[name])
         self.device = device
         self.ratio = synth.ratio_schedule(w)
+        if layers > 0:            # profiling aid: the first `layers` layers of the schedule only
+            self.ratio = self.ratio[:layers]
+            w["n_layers"] = layers
+        if decode_steps >= 0:
+            w["max_new_tokens"] = decode_steps
         self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio))
         self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
         B, N, Hq, Hkv, D = w["batch"], w["prompt_len"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
@@ -193,7 +198,7 @@ def run_ours(args, rank, world, local_rank):
     from paper_2405_12532_b200 import binding as pb
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
-    wl = Workload(args.workload, device)
+    wl = Workload(args.workload, device, layers=args.layers, decode_steps=args.decode_steps)
     w = wl.w
     nL = w["n_layers"]
     hbm, tf_burst, tf_sust, peak_src = measured_peaks()
@@ -414,6 +419,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first LAYERS layers")
+    ap.add_argument("--decode-steps", type=int, default=-1, help="profiling aid: override the decode steps")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -309,22 +309,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // S = Q K^T, both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
+      // operand descriptors are built once; a k-step only adds a constant to the start-address field
+      const uint64_t dq0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024), dq1 = smem_desc_sw128(smem_u32(sm.q[1]), 16, 1024);
+      const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
+      const uint64_t dv0 = smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
+      const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
       auto issue_s = [&](int w, int st) {
-        const uint32_t qa = smem_u32(sm.q[w]), ka = smem_u32(sm.k[st]);
+        const uint64_t qd = w ? dq1 : dq0, kd = st ? dk1 : dk0;
+        const uint32_t d_tmem = tmem + w * kTile;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          mma_ss(tmem + w * kTile, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_s,
-                 kk > 0);
+          const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+          mma_ss(d_tmem, qd + off, kd + off, idesc_s, kk > 0);
         }
         mma_commit(&sm.s_full[w]);
       };
       auto issue_pv = [&](int w, int st, bool accumulate) {
-        const uint32_t va = smem_u32(sm.v[st]);
+        const uint64_t vd = st ? dv1 : dv0;
+        const uint32_t d_tmem = tmem + (2 + w) * kTile, p_tmem = tmem + w * kTile;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
-          mma_ts(tmem + (2 + w) * kTile, tmem + w * kTile + kk * 8,
-                 smem_desc_sw128(va + kk * 2048, kHalfBytes, 1024), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
+          mma_ts(d_tmem, p_tmem + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
         mma_commit(&sm.o_done[w]);
       };
       bool ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, code);
@@ -380,20 +385,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       ok = mbar_wait(&sm.s_full[w], j & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[128];
+      const bool diag = j == nkt_w - 1;     // diagonal tile: key 128 j + col is visible iff col <= lim
+      const int lim = i - j * kTile;
+      // pass 1: the row maximum (S is read twice from tensor memory rather than held in 128 registers)
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, s + ch * 32);
-      tmem_wait_ld();
-      if (j == nkt_w - 1) {            // diagonal tile: key 128 j + col is visible iff it is <= i
-        const int lim = i - j * kTile;
+      for (int half = 0; half < 2; ++half) {
+        uint32_t ra[32], rb[32];
+        tmem_ld32(s_addr + half * 64, ra);
+        tmem_ld32(s_addr + half * 64 + 32, rb);
+        tmem_wait_ld();
+        if (diag) {
 #pragma unroll
-        for (int col = 0; col < 128; ++col)
-          if (col > lim) s[col] = 0xff800000u;   // -inf
+          for (int col = 0; col < 32; ++col) {
+            if (half * 64 + col > lim) ra[col] = 0xff800000u;
+            if (half * 64 + 32 + col > lim) rb[col] = 0xff800000u;
+          }
+        }
+#pragma unroll
+        for (int col = 0; col < 32; col += 4) {
+          mx0 = max3(mx0, __uint_as_float(ra[col]), __uint_as_float(ra[col + 1]));
+          mx1 = max3(mx1, __uint_as_float(ra[col + 2]), __uint_as_float(ra[col + 3]));
+          mx2 = max3(mx2, __uint_as_float(rb[col]), __uint_as_float(rb[col + 1]));
+          mx3 = max3(mx3, __uint_as_float(rb[col + 2]), __uint_as_float(rb[col + 3]));
+        }
       }
-      float mx = __uint_as_float(s[0]);
-#pragma unroll
-      for (int col = 1; col < 128; ++col) mx = fmaxf(mx, __uint_as_float(s[col]));
-      mx *= sc2;
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
       const bool need = mx > m_used + kRescaleStep;      // also true on the first tile (m_used = -inf)
       if (j > 0 && __any_sync(0xffffffffu, need)) {
         // O of this tile must hold every PV issued so far before it is rescaled
@@ -413,14 +430,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         l *= f;
       }
       if (need) m_used = mx;
+      // pass 2: P = exp2(S * scale - m), written over S as bf16, 32 columns at a time; the next
+      // 32 columns are in flight while these are exponentiated
       float part[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t buf[2][32];
+      tmem_ld32(s_addr, buf[0]);
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
+        uint32_t* cur = buf[ch & 1];
+        tmem_wait_ld();
+        if (ch < 3) tmem_ld32(s_addr + (ch + 1) * 32, buf[(ch + 1) & 1]);
+        if (diag) {
+#pragma unroll
+          for (int col = 0; col < 32; ++col)
+            if (ch * 32 + col > lim) cur[col] = 0xff800000u;
+        }
         uint32_t p[16];
 #pragma unroll
         for (int c2 = 0; c2 < 16; ++c2) {
-          const float p0 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2]), sc2, -m_used));
-          const float p1 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2 + 1]), sc2, -m_used));
+          const float p0 = ex2(fmaf(__uint_as_float(cur[2 * c2]), sc2, -m_used));
+          const float p1 = ex2(fmaf(__uint_as_float(cur[2 * c2 + 1]), sc2, -m_used));
           part[c2 & 1] += p0;
           part[2 + (c2 & 1)] += p1;
           p[c2] = pack_bf16(p0, p1);

@@ -136,6 +136,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+// Same load, and a zero produced inside the same asm statement. Arithmetic that takes the zero as an
+// operand cannot be scheduled ahead of the load, which lets a caller put the load of the NEXT chunk
+// in flight before the arithmetic on the current one starts.
+__device__ __forceinline__ uint32_t tmem_ld32_zero(uint32_t taddr, uint32_t* r) {
+  uint32_t zero;
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
+      "mov.b32 %32, 0;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+        "=r"(zero)
+      : "r"(taddr)
+      : "memory");
+  return zero;
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -207,6 +226,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Host: a 4-D tensor map over a [B, n, H, D] bf16 tensor with element strides
 // (sb, sn, sh, 1), box = 64 elements of D x `box_rows` rows of one head, 128-byte swizzle.
+bool tensor_maps_available();   // the driver's tensor-map encoder could be resolved
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int B, int n, int H, int D, int64_t sb, int64_t sn,
                           int64_t sh, int box_rows);
 

@@ -2,19 +2,22 @@
 // Algorithm 1, "compute attention weights of KV", and the attention output.
 //
 // A CTA owns 256 consecutive query rows of one (sequence, head): two 128-row
-// tiles that share every K and V tile it loads.
-//   warps 0-15  softmax: tile w = warp / 8; the two warps that serve the same 32 rows
-//               (warp % 4 = TMEM lane quarter) split the 128 keys of a tile in halves
-//   warp 16     MMA issue for both tiles (one lane)
-//   warp 17     TMA loads (one lane)
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P
-// (bf16) overwrites the first 64 columns of its S. Per tile and key tile j the
-// order is S(j) -> softmax -> PV(j) -> S(j+1); the issuing thread alternates
-// between the tiles (PV0 S0 PV1 S1), so one tile's softmax overlaps the
-// other's tensor work. The running maximum used in the exponent is
-// only raised when the row maximum has grown by more than 2^8, which keeps
-// rescaling of O (a TMEM round trip) rare; the final normalisation uses the same
-// maximum, so the result is the exact softmax.
+// tiles that share every K and V tile it loads (TMA, 128 keys per tile, two
+// stages each).
+//   warps 0-3 / 4-7   softmax of tile 0 / 1, thread = one query row
+//   warp 8 / 9        MMA issue for tile 0 / 1 (one lane each)
+//   warp 10           TMA loads (one lane)
+// The keys are consumed in half-steps of 64. Tensor memory, per tile 256 of the
+// 512 columns: two S buffers of 64 fp32 columns and O (128 columns); P (bf16)
+// overwrites the first 32 columns of its S buffer. Because S is double
+// buffered, the issuing thread runs S(t+1) while the softmax of half-step t is
+// at work, and PV(t) follows as soon as P(t) is there:
+//     S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
+// so the tensor pipe and the softmax threads only meet through the two-deep
+// buffer, not once per step. The running maximum used in the exponent is only
+// raised when the row maximum has grown by more than 2^8, which keeps rescaling
+// of O (a TMEM round trip) rare; the final normalisation uses the same maximum,
+// so the result is the exact softmax.
 #include <cuda_bf16.h>
 
 #include "pyr_internal.h"
@@ -27,26 +30,23 @@ using namespace tc;
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int kTile = 128;
-constexpr int kHalfBytes = kTile * 128;     // one [128 rows x 64 bf16] swizzled half tile
+constexpr int kTile = 128;                  // query rows per tile, keys per K/V tile
+constexpr int kHalf = 64;                   // keys per half-step
+constexpr int kHalfBytes = kTile * 128;     // one [128 rows x 64 bf16] swizzled half tile (half of D)
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128 x 128] bf16 tile = two halves along D
-constexpr int kSoftmaxWarps = 16;
-constexpr int kThreads = (kSoftmaxWarps + 2) * 32;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
 constexpr float kRescaleStep = 8.0f;
 
 struct AttnSmem {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
-  float xmax[2][2][2][kTile];   // [tile][step parity][key half][row]
-  float xsum[2][2][kTile];      // [tile][key half][row]
-  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_ready[2], o_done[2];
+  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2];   // [tile][S buffer]
   uint32_t tmem_base;
   int abort_flag;
 };
-
-__device__ __forceinline__ void pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
-__device__ __forceinline__ void pair_arrive(int id) { asm volatile("bar.arrive %0, 64;" ::"r"(id) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -72,12 +72,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     mbar_init(&sm.q_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.k_full[i], 1);
-      mbar_init(&sm.k_empty[i], 1);
+      mbar_init(&sm.k_empty[i], users);
       mbar_init(&sm.v_full[i], 1);
-      mbar_init(&sm.v_empty[i], 1);
-      mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.p_ready[i], 2 * kTile);
+      mbar_init(&sm.v_empty[i], users);
       mbar_init(&sm.o_done[i], 1);
+      for (int bf = 0; bf < 2; ++bf) {
+        mbar_init(&sm.s_full[i][bf], 1);
+        mbar_init(&sm.p_ready[i][bf], kTile);
+      }
     }
     sm.abort_flag = 0;
     fence_barrier_init();
@@ -92,7 +94,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t tmem = sm.tmem_base;
   const int code = PYR_ERR_TIMEOUT;
 
-  if (warp == kSoftmaxWarps + 1) {
+  if (warp == kSoftmaxWarps + 2) {
     // ---------------------------------------------------------------- TMA loads
     if (lane == 0) {
       prefetch_tensormap(&map_q);
@@ -120,190 +122,142 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     __syncwarp();
   } else if (warp >= kSoftmaxWarps) {
-    // ---------------------------------------------------------------- MMA issue (one thread, both tiles)
-    if (lane == 0 && warp == kSoftmaxWarps) {
-      constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // S = Q K^T, both K-major
+    // ---------------------------------------------------------------- MMA issue, one thread per tile
+    const int w = warp - kSoftmaxWarps;
+    const int T = 2 * (w ? nkt1 : nkt0);           // half-steps of this tile
+    if (lane == 0 && T > 0) {
+      constexpr uint32_t idesc_s = idesc_bf16(kTile, kHalf, false, false);   // S = Q K^T (64 keys), both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
       // operand descriptors are built once; a k-step only adds a constant to the start-address field
-      const uint64_t dq0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024), dq1 = smem_desc_sw128(smem_u32(sm.q[1]), 16, 1024);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[w]), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
       const uint64_t dv0 = smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
-      auto issue_s = [&](int w, int st) {
-        const uint64_t qd = w ? dq1 : dq0, kd = st ? dk1 : dk0;
-        const uint32_t d_tmem = tmem + w * kTile;
+      const uint32_t t_base = tmem + w * 256, o_tmem = t_base + 128;
+      bool ok = true;
+      // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
+      auto issue_s = [&](int t) {
+        const int j = t >> 1, st = j & 1, bf = t & 1;
+        if (bf == 0) {
+          ok = mbar_wait(&sm.k_full[st], (j >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) return;
+          tc_fence_after();
+        }
+        const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-          mma_ss(d_tmem, qd + off, kd + off, idesc_s, kk > 0);
+          mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
         }
-        mma_commit(&sm.s_full[w]);
+        mma_commit(&sm.s_full[w][bf]);
+        if (bf == 1) mma_commit(&sm.k_empty[st]);
       };
-      auto issue_pv = [&](int w, int st, bool accumulate) {
-        const uint64_t vd = st ? dv1 : dv0;
-        const uint32_t d_tmem = tmem + (2 + w) * kTile, p_tmem = tmem + w * kTile;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
-          mma_ts(d_tmem, p_tmem + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
-        mma_commit(&sm.o_done[w]);
-      };
-      // Order per key tile j: PV0(j) S0(j+1) PV1(j) S1(j+1). While one tile's softmax runs, the
-      // other tile's two groups keep the tensor pipe busy.
-      bool ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, code);
-      if (ok) ok = mbar_wait(&sm.k_full[0], 0, abort_flag, a.status, code);
-      if (ok) {
-        tc_fence_after();
-        issue_s(0, 0);
-        if (valid1) issue_s(1, 0);
-        mma_commit(&sm.k_empty[0]);
-      }
-      const int last_w = valid1 ? 1 : 0;
-      for (int j = 0; j < nkt && ok; ++j) {
-        const int st = j & 1, st1 = (j + 1) & 1;
-        ok = mbar_wait(&sm.v_full[st], (j >> 1) & 1, abort_flag, a.status, code);
+      ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, code);
+      if (ok) issue_s(0);
+      if (ok) issue_s(1);
+      for (int t = 0; t < T && ok; ++t) {
+        const int j = t >> 1, st = j & 1, bf = t & 1;
+        if (bf == 0) ok = mbar_wait(&sm.v_full[st], (j >> 1) & 1, abort_flag, a.status, code);
+        if (ok) ok = mbar_wait(&sm.p_ready[w][bf], (t >> 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
-        bool k_next_ready = false;
-        for (int w = 0; w < 2 && ok; ++w) {
-          const int nkt_w = w ? nkt1 : nkt0;
-          if (j < nkt_w) {
-            ok = mbar_wait(&sm.p_ready[w], j & 1, abort_flag, a.status, code);
-            if (!ok) break;
-            tc_fence_after();
-            issue_pv(w, st, j > 0);
-          }
-          if (w == last_w) mma_commit(&sm.v_empty[st]);
-          if (j + 1 < nkt_w) {
-            if (!k_next_ready) {
-              ok = mbar_wait(&sm.k_full[st1], ((j + 1) >> 1) & 1, abort_flag, a.status, code);
-              if (!ok) break;
-              k_next_ready = true;
-              tc_fence_after();
-            }
-            issue_s(w, st1);
-          }
-          if (w == last_w && j + 1 < nkt) mma_commit(&sm.k_empty[st1]);
-        }
+        tc_fence_after();
+        const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
+          mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+                 (t > 0 || kk > 0) ? 1u : 0u);
+        mma_commit(&sm.o_done[w]);
+        if (bf == 1) mma_commit(&sm.v_empty[st]);
+        if (t + 2 < T) issue_s(t + 2);
       }
     }
     __syncwarp();
   } else {
-    // ---------------------------------------------------------------- softmax
-    const int w = warp >> 3;                       // query tile
-    const int hh = (warp >> 2) & 1;                // which 64 keys of a 128-key tile
-    const int quarter = warp & 3;                  // TMEM lane quarter = rows 32 * quarter ...
-    const int row = quarter * 32 + lane;
-    const int i = r0 + w * kTile + row;            // query row of this thread
-    const int bar_id = 1 + w * 4 + quarter;        // named barrier of the two warps that share these rows
-    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + w * kTile;            // S of the tile, column 0
-    const uint32_t my_s = s_addr + hh * 64;                          // my 64 key columns
-    const uint32_t my_p = s_addr + hh * 32;                          // where their bf16 P goes
-    const uint32_t my_o = tmem + lane_base + (2 + w) * kTile + hh * 64;   // my 64 columns of O
-    const int nkt_w = w ? nkt1 : nkt0;
+    // ---------------------------------------------------------------- softmax, thread = query row
+    const int w = warp >> 2;
+    const int row = threadIdx.x & (kTile - 1);
+    const int i = r0 + w * kTile + row;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_base = tmem + lane_base + w * 256;
+    const uint32_t o_addr = t_base + 128;
+    const int T = 2 * (w ? nkt1 : nkt0);
     const float sc2 = a.scale * kLog2e;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < nkt_w && ok; ++j) {
-      ok = mbar_wait(&sm.s_full[w], j & 1, abort_flag, a.status, code);
+    for (int t = 0; t < T && ok; ++t) {
+      const int bf = t & 1;
+      const uint32_t s_addr = t_base + bf * kHalf;
+      ok = mbar_wait(&sm.s_full[w][bf], (t >> 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
-      const bool diag = j == nkt_w - 1;            // diagonal tile: key 128 j + col is visible iff col <= lim
-      const int lim = i - j * kTile - hh * 64;     // in my own column numbering
-      // pass 1: maximum over my 64 keys, then over the partner's
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-      {
-        uint32_t ra[32], rb[32];
-        tmem_ld32(my_s, ra);
-        tmem_ld32(my_s + 32, rb);
-        tmem_wait_ld();
-        if (diag) {
+      uint32_t s[64];
+      tmem_ld32(s_addr, s);
+      tmem_ld32(s_addr + 32, s + 32);
+      tmem_wait_ld();
+      if (t >= T - 2) {                 // inside the diagonal key tile: key 64 t + col is visible iff col <= lim
+        const int lim = i - t * kHalf;
 #pragma unroll
-          for (int col = 0; col < 32; ++col) {
-            if (col > lim) ra[col] = 0xff800000u;
-            if (32 + col > lim) rb[col] = 0xff800000u;
-          }
-        }
-#pragma unroll
-        for (int col = 0; col < 32; col += 4) {
-          mx0 = max3(mx0, __uint_as_float(ra[col]), __uint_as_float(ra[col + 1]));
-          mx1 = max3(mx1, __uint_as_float(ra[col + 2]), __uint_as_float(ra[col + 3]));
-          mx2 = max3(mx2, __uint_as_float(rb[col]), __uint_as_float(rb[col + 1]));
-          mx3 = max3(mx3, __uint_as_float(rb[col + 2]), __uint_as_float(rb[col + 3]));
-        }
+        for (int col = 0; col < 64; ++col)
+          if (col > lim) s[col] = 0xff800000u;   // -inf
       }
-      const float own = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      sm.xmax[w][j & 1][hh][row] = own;
-      pair_sync(bar_id);
-      const float mx = fmaxf(own, sm.xmax[w][j & 1][hh ^ 1][row]) * sc2;   // finite: key 128 j is visible
-      const bool need = mx > m_used + kRescaleStep;      // also true on the first tile (m_used = -inf)
-      if (j > 0 && __any_sync(0xffffffffu, need)) {
-        // O of this tile must hold every PV issued so far before it is rescaled; both partner
-        // warps hold the same rows and take this branch together
-        ok = mbar_wait(&sm.o_done[w], (j - 1) & 1, abort_flag, a.status, code);
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int col = 0; col < 64; col += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
+      }
+      // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
+      const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
+      if (t > 0 && __any_sync(0xffffffffu, need)) {
+        // O must hold every PV issued so far before it is rescaled
+        ok = mbar_wait(&sm.o_done[w], (t - 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
         tc_fence_after();
         const float f = need ? ex2(m_used - mx) : 1.f;
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
+        for (int ch = 0; ch < 4; ++ch) {
           uint32_t o[32];
-          tmem_ld32(my_o + ch * 32, o);
+          tmem_ld32(o_addr + ch * 32, o);
           tmem_wait_ld();
 #pragma unroll
           for (int col = 0; col < 32; ++col) o[col] = __float_as_uint(__uint_as_float(o[col]) * f);
-          tmem_st32(my_o + ch * 32, o);
+          tmem_st32(o_addr + ch * 32, o);
         }
         l *= f;
       }
       if (need) m_used = mx;
-      // pass 2: P = exp2(S * scale - m) over my 64 keys, written over S as bf16. P of keys
-      // 64..127 lands on S columns 32..63, which the partner (keys 0..63) reads: it signals
-      // once it holds them in registers, and the upper half waits for that before storing.
+      const float neg_m = -m_used;
       float part[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t buf[2][32];
-      tmem_ld32(my_s, buf[0]);
 #pragma unroll
       for (int ch = 0; ch < 2; ++ch) {
-        uint32_t* cur = buf[ch];
-        tmem_wait_ld();
-        uint32_t zero = 0u;
-        if (ch == 0) zero = tmem_ld32_zero(my_s + 32, buf[1]);   // in flight during this chunk's arithmetic
-        if (ch == 1 && hh == 0) pair_arrive(bar_id);
-        const float neg_m = __uint_as_float(zero) - m_used;
-        if (diag) {
-#pragma unroll
-          for (int col = 0; col < 32; ++col)
-            if (ch * 32 + col > lim) cur[col] = 0xff800000u;
-        }
         uint32_t p[16];
 #pragma unroll
         for (int c2 = 0; c2 < 16; ++c2) {
-          const float p0 = ex2(fmaf(__uint_as_float(cur[2 * c2]), sc2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(cur[2 * c2 + 1]), sc2, neg_m));
+          const float p0 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2]), sc2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2 + 1]), sc2, neg_m));
           part[c2 & 1] += p0;
           part[2 + (c2 & 1)] += p1;
           p[c2] = pack_bf16(p0, p1);
         }
-        if (ch == 0 && hh == 1) pair_sync(bar_id);
-        tmem_st16(my_p + ch * 16, p);
+        tmem_st16(s_addr + ch * 16, p);
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&sm.p_ready[w]);
+      mbar_arrive(&sm.p_ready[w][bf]);
       l += (part[0] + part[1]) + (part[2] + part[3]);
     }
-    // row sum over both key halves, then my 64 columns of the output
-    sm.xsum[w][hh][row] = l;
-    pair_sync(bar_id);
-    const float l_all = l + sm.xsum[w][hh ^ 1][row];
-    if (ok && nkt_w > 0) ok = mbar_wait(&sm.o_done[w], (nkt_w - 1) & 1, abort_flag, a.status, code);
-    if (ok && nkt_w > 0) {
+    if (ok && T > 0) ok = mbar_wait(&sm.o_done[w], (T - 1) & 1, abort_flag, a.status, code);
+    if (ok && T > 0) {
       tc_fence_after();
-      const float inv = 1.f / l_all;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.out) + b * a.osb + h * a.osh + (int64_t)i * a.osn + hh * 64;
+      const float inv = 1.f / l;
+      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.out) + b * a.osb + h * a.osh + (int64_t)i * a.osn;
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
+      for (int ch = 0; ch < 4; ++ch) {
         uint32_t o[32];
-        tmem_ld32(my_o + ch * 32, o);
+        tmem_ld32(o_addr + ch * 32, o);
         tmem_wait_ld();
         if (i < n) {
 #pragma unroll
@@ -317,7 +271,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
         }
       }
-      if (hh == 0 && i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l_all)) * kLn2;
+      if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
     }
   }
   tc_fence_before();

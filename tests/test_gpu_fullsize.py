@@ -1,0 +1,124 @@
+"""GPU parity at the full sizes of the workloads, in the launch configuration the
+benchmark times: one layer of the schedule at the full batch, checked against the
+oracle on sampled (sequence, group) pairs and sampled rows. Every (layer,
+sequence, group) call of an attention stack is independent of the others (its
+inputs are drawn at the surviving length), so a sample is a complete check of
+the calls it covers."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_12532_b200 import binding as pb
+from paper_2405_12532_b200 import synth
+from parity_util import check_kept, one_layer_cache, tol_for
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+CASES = [
+    # workload, layers of its schedule to run, (sequence, group) samples per layer
+    ("7b_stack_8x2k", [1, 16, 31], 3),
+    ("7b_64x2k", [1, 31], 2),
+    ("13b_stack_32x4k", [1, 39], 2),
+    ("70b_gqa_16x8k", [1, 79], 2),
+]
+
+
+def _sample_pairs(B, G, count, seed):
+    rng = np.random.default_rng(seed)
+    pairs = {(0, 0), (B - 1, G - 1)}
+    while len(pairs) < count + 2:
+        pairs.add((int(rng.integers(B)), int(rng.integers(G))))
+    return sorted(pairs)
+
+
+@pytest.mark.parametrize("name,layers,nsamp", CASES, ids=[c[0] for c in CASES])
+def test_full_size_layer_against_oracle(name, layers, nsamp):
+    w = dict(synth.CONFIGS[name])
+    ratio = synth.ratio_schedule(w)
+    budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
+    B, Hq, Hkv, D, L, G = w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["recent_len"], w["sel_groups"]
+    rep = Hq // Hkv
+    heads_per_group = Hq // G
+    tol = tol_for(w["dtype"])
+    w1 = dict(w, max_new_tokens=2)
+    ties = exact = 0
+    for l in layers:
+        bud = budgets[l]
+        n, k, c = bud["n_in"], bud["k"], bud["c"]
+        cache = one_layer_cache(w1, n, k)
+        assert cache.layer_info(0)["k_ctx"] == k
+        Q, K, V = synth.stack_layer_inputs(w, l, n, device=DEV)
+        out = torch.empty_like(Q)
+        cache.prefill_layer(0, Q, K, V, out)
+        torch.cuda.synchronize()
+        lse = cache.lse(0)
+        score = cache.scores(0).clone()
+        O0 = out.clone() if G != 1 else None
+        if G == 1:
+            hidden = w.get("hidden", Hq * D)
+            gen = torch.Generator(device=DEV); gen.manual_seed(l)
+            rows = torch.randn(B, n, hidden, generator=gen, device=DEV).to(torch.bfloat16)
+            rows0 = rows.clone()
+            n_out = cache.select_compact(0, K, V, rows, hidden, n * hidden, hidden, 0)
+        else:
+            n_out = cache.select_compact(0, K, V, out, rep * D, out.stride(0), out.stride(1), rep * D)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        assert n_out == bud["n_out"]
+        kept_all, pos_all = cache.kept(0)
+        Kc, Vc = cache.kv(0)
+        rng = np.random.default_rng(100 + l)
+        for (b, g) in _sample_pairs(B, G, nsamp, seed=l):
+            heads = list(range(g * heads_per_group, (g + 1) * heads_per_group))
+            # scores of the group from the recent rows of each of its heads
+            E = np.zeros((len(heads), c))
+            recent = np.arange(c, n)
+            wts = oracle.recent_weights(L)
+            for hi, h in enumerate(heads):
+                A, lse_ref = oracle.attention_weights(synth.widen(Q[b, :, h]), synth.widen(K[b, :, h // rep]),
+                                                      oracle.softmax_scale_default(D), recent)
+                E[hi] = oracle.ensemble_score(A, L, wts)
+                assert np.abs(synth.widen(lse[b, h, c:]) - lse_ref).max() <= 2e-3
+            sc_ref = oracle.pooled_scores(E, 1)[0]
+            np.testing.assert_allclose(synth.widen(score[b, g]), sc_ref, rtol=2e-3, atol=1e-30)
+            kept = kept_all[b, g].cpu().numpy()
+            res = check_kept(kept, sc_ref, k, n, L)
+            ties += res == "tie"; exact += res == "exact"
+            np.testing.assert_array_equal(pos_all[b, g].cpu().numpy(), kept)
+            idx = torch.from_numpy(kept).to(DEV).long()
+            # attention output on sampled rows of one head of the group
+            h = heads[int(rng.integers(len(heads)))]
+            rows_s = np.sort(rng.choice(n, size=48, replace=False))
+            rows_s[0], rows_s[-1] = 0, n - 1
+            A, _ = oracle.attention_weights(synth.widen(Q[b, :, h]), synth.widen(K[b, :, h // rep]),
+                                            oracle.softmax_scale_default(D), rows_s)
+            O_ref = A @ synth.widen(V[b, :, h // rep])
+            O_src = out if G == 1 else O0
+            assert np.abs(synth.widen(O_src[b, torch.from_numpy(rows_s).to(DEV), h]) - O_ref).max() <= tol
+            # gathers are byte-exact
+            for kvh in ([h // rep] if G != 1 else [int(rng.integers(Hkv))]):
+                assert torch.equal(Kc[b, kvh, :n_out], K[b, idx, kvh])
+                assert torch.equal(Vc[b, kvh, :n_out], V[b, idx, kvh])
+            if G == 1:
+                assert torch.equal(rows[b, :n_out], rows0[b, idx])
+            else:
+                assert torch.equal(out[b, :n_out, g * rep:(g + 1) * rep], O0[b, idx, g * rep:(g + 1) * rep])
+        # two decode steps over this layer's cache, checked on sampled (sequence, head) pairs
+        for t in range(2):
+            q, kn, vn = synth.decode_step_inputs(w, l, t, device=DEV)
+            o = torch.empty_like(q)
+            ln = cache.layer_info(0)["len_now"]
+            cache.decode_attn(0, q, kn, vn, o)
+            torch.cuda.synchronize()
+            for (b, g) in _sample_pairs(B, Hkv, 2, seed=7 + t):
+                Kb, Vb = synth.widen(Kc[b, g:g + 1, :ln]), synth.widen(Vc[b, g:g + 1, :ln])
+                qs = synth.widen(q[b, g * rep:(g + 1) * rep])
+                want, _, _ = oracle.decode_attention(qs, Kb, Vb, synth.widen(kn[b, g:g + 1]), synth.widen(vn[b, g:g + 1]))
+                assert np.abs(synth.widen(o[b, g * rep:(g + 1) * rep]) - want).max() <= tol
+            assert torch.equal(Kc[:, :, ln], kn) and torch.equal(Vc[:, :, ln], vn)
+        cache.close()
+        del Q, K, V, out, cache
+        torch.cuda.empty_cache()
+    print(f"{name}: {exact} selections identical to the oracle's, {ties} differ only within the 1e-6 tie band")

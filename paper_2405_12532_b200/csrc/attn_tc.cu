@@ -211,10 +211,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
       const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
-      if (t > 0 && __any_sync(0xffffffffu, need)) {
-        // O must hold every PV issued so far before it is rescaled
+      // A parity wait is only meaningful one phase behind the barrier, so o_done is followed on
+      // every half-step (PV(t-1) was issued a whole softmax ago: this wait is normally free).
+      if (t > 0) {
         ok = mbar_wait(&sm.o_done[w], (t - 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
+      }
+      if (t > 0 && __any_sync(0xffffffffu, need)) {
+        // O holds every PV issued so far: it can be rescaled
         tc_fence_after();
         const float f = need ? ex2(m_used - mx) : 1.f;
 #pragma unroll

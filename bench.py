@@ -98,7 +98,7 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs and the call sequence of one step."""
 
-    def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1):
+    def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1, batch: int = 0):
         from paper_2405_12532_b200 import binding as pb
         self.pb = pb
         self.name = name
@@ -110,6 +110,8 @@ class Workload:
             w["n_layers"] = layers
         if decode_steps >= 0:
             w["max_new_tokens"] = decode_steps
+        if batch > 0:             # profiling aid: a smaller batch keeps an ncu capture small
+            w["batch"] = batch
         self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio))
         self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
         B, N, Hq, Hkv, D = w["batch"], w["prompt_len"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
@@ -198,7 +200,7 @@ def run_ours(args, rank, world, local_rank):
     from paper_2405_12532_b200 import binding as pb
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
-    wl = Workload(args.workload, device, layers=args.layers, decode_steps=args.decode_steps)
+    wl = Workload(args.workload, device, layers=args.layers, decode_steps=args.decode_steps, batch=args.batch)
     w = wl.w
     nL = w["n_layers"]
     hbm, tf_burst, tf_sust, peak_src = measured_peaks()
@@ -421,6 +423,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first LAYERS layers")
     ap.add_argument("--decode-steps", type=int, default=-1, help="profiling aid: override the decode steps")
+    ap.add_argument("--batch", type=int, default=0, help="profiling aid: override the batch size")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

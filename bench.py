@@ -30,6 +30,9 @@ import torch
 from paper_2405_12532_b200 import synth
 
 METRIC = "prefill tokens/s + decode tokens/s at 7B shapes 64x2k"
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch divided by its algorithmic bytes
+# (542.47 MB / 537.13 MB in profiles/decode_kernel_7b_2k_batch16.txt). Set to None when the kernel changes.
+DECODE_TRAFFIC_RATIO = 542.47 / 537.13
 DEFAULT_WORKLOAD = "7b_64x2k"
 
 
@@ -258,7 +261,10 @@ def run_ours(args, rank, world, local_rank):
     if T > 0:
         ach = K * dec_bytes / t_dec / 1e9
         roof_dec = {"kernel": "decode_kernel", "bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s",
-                    "frac": ach / hbm, "traffic": None, "peak_source": f"of {peak_src}",
+                    "frac": ach / hbm, "traffic": DECODE_TRAFFIC_RATIO * dec_bytes / dec_launches,
+                    "traffic_note": "dram read+write bytes per launch, scaled from one ncu capture at batch 16 "
+                                    "(profiles/decode_kernel_7b_2k_batch16.txt) by the rows streamed",
+                    "peak_source": f"of {peak_src}",
                     "launches": K * dec_launches, "avg_launch_us": t_dec / (K * dec_launches) * 1e6,
                     "algorithmic_bytes_per_launch": dec_bytes / dec_launches}
     ach_tf = K * wl.prefill_flops() / t_attn / 1e12

@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 
 import torch
 
+from paper_2405_12532_b200 import dist as pdist
 from paper_2405_12532_b200 import synth
 
 METRIC = "prefill tokens/s + decode tokens/s at 7B shapes 64x2k"
@@ -209,9 +210,7 @@ def run_ours(args, rank, world, local_rank):
     hbm, tf_burst, tf_sust, peak_src = measured_peaks()
 
     def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
+        pdist.barrier(world)
 
     for _ in range(args.warmup):
         wl.prefill(); wl.decode()
@@ -240,14 +239,11 @@ def run_ours(args, rank, world, local_rank):
     t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
     t_attn = sum(e[0].elapsed_time(e[1]) for st in ev for e in st) / 1e3
     t_sel = sum(e[1].elapsed_time(e[2]) for st in ev for e in st) / 1e3
-    times = torch.tensor([t_pre, t_dec, t_attn, t_sel, t_pre + t_dec], dtype=torch.float64, device=device)
-    if world > 1:
-        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
-    t_pre, t_dec, t_attn, t_sel, t_all = [float(x) for x in times.tolist()]
+    t_pre, t_dec, t_attn, t_sel, t_all = pdist.max_over_ranks([t_pre, t_dec, t_attn, t_sel, t_pre + t_dec], world, device)
 
     K = args.steps
     B, N, T = w["batch"], w["prompt_len"], w["max_new_tokens"]
-    prefill_tps = world * K * B * N / t_pre
+    prefill_tps = pdist.whole_job_rate(K * B * N, world, t_pre)
     decode_tps = world * K * B * T / t_dec if T > 0 and t_dec > 0 else None
 
     # ---- end to end: host buffers, copies inside the timed region
@@ -348,10 +344,7 @@ def run_e2e(wl, args, barrier, world):
         step(True)
     e1.record()
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1) / 1e3], dtype=torch.float64, device=wl.device)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    t = float(t.item())
+    t = pdist.max_over_ranks([e0.elapsed_time(e1) / 1e3], world, wl.device)[0]
     B, N, T = w["batch"], w["prompt_len"], w["max_new_tokens"]
     return {"value": world * steps * B * (N + T) / t, "unit": "tokens/s (prompt + generated, whole step from host buffers)",
             "steps": steps, "ms_per_step": t / steps * 1e3,
@@ -438,8 +431,7 @@ def main():
         run_reference(args, rank, world)
         return
     if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        pdist.init("nccl", torch.device("cuda", local_rank))
     try:
         run_ours(args, rank, world, local_rank)
     finally:

@@ -1,9 +1,11 @@
 // tcgen05 causal attention of the prefill step (bf16, head_dim 128):
 // Algorithm 1, "compute attention weights of KV", and the attention output.
 //
-// A CTA owns 256 consecutive query rows of one (sequence, head): two 128-row
-// tiles that share every K and V tile it loads (TMA, 128 keys per tile, two
-// stages each).
+// A CTA owns one (sequence, head) and walks its query rows in blocks of 256:
+// two 128-row tiles that share every K and V tile the CTA loads (TMA, 128 keys
+// per tile, two stages each). Because the CTA stays on the head, the loads, the
+// first MMAs and the output epilogue of consecutive blocks overlap instead of
+// paying a prologue per block, and every CTA of the grid does the same work.
 //   warps 0-3 / 4-7   softmax of tile 0 / 1, thread = one query row
 //   warp 8 / 9        MMA issue for tile 0 / 1 (one lane each)
 //   warp 10           TMA loads (one lane)
@@ -13,11 +15,13 @@
 // buffered, the issuing thread runs S(t+1) while the softmax of half-step t is
 // at work, and PV(t) follows as soon as P(t) is there:
 //     S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
-// so the tensor pipe and the softmax threads only meet through the two-deep
-// buffer, not once per step. The running maximum used in the exponent is only
-// raised when the row maximum has grown by more than 2^8, which keeps rescaling
-// of O (a TMEM round trip) rare; the final normalisation uses the same maximum,
-// so the result is the exact softmax.
+// The running maximum used in the exponent is only raised when the row maximum
+// has grown by more than 2^8, which keeps rescaling of O (a TMEM round trip)
+// rare; the final normalisation uses the same maximum, so the result is the
+// exact softmax.
+//
+// All mbarriers live across blocks, so every role counts the phases it has
+// consumed (a parity wait is only valid one phase behind the barrier).
 #include <cuda_bf16.h>
 
 #include "pyr_internal.h"
@@ -42,11 +46,25 @@ struct AttnSmem {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
-  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t q_full[2], q_empty[2];                    // per tile
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2];   // [tile][S buffer]
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// Geometry of one 256-row block of the head.
+struct Block {
+  int r0, nkt0, nkt1, nkt;   // first row; key tiles of tile 0 / tile 1 (0 = tile absent) / loaded
+};
+__device__ __forceinline__ Block block_of(int blk, int n) {
+  Block b;
+  b.r0 = blk * 2 * kTile;
+  b.nkt0 = 2 * blk + 1;                               // causal: the diagonal tile is the last one
+  b.nkt1 = (b.r0 + kTile < n) ? 2 * blk + 2 : 0;
+  b.nkt = b.nkt1 ? b.nkt1 : b.nkt0;
+  return b;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -54,27 +72,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-  const int pair = gridDim.x - 1 - blockIdx.x;     // longest rows first
-  const int h = blockIdx.y, b = blockIdx.z;
+  const int h = blockIdx.x, b = blockIdx.y;
   const int g = h / (a.Hq / a.Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = a.n;
-  const int r0 = pair * 2 * kTile;
-  const bool valid1 = r0 + kTile < n;
-  const int nkt0 = 2 * pair + 1;                   // key tiles of query tile 0 (diagonal last)
-  const int nkt1 = valid1 ? 2 * pair + 2 : 0;
-  const int nkt = valid1 ? nkt1 : nkt0;
-  const int users = valid1 ? 2 : 1;                // tiles that read each K / V stage
+  const int nblk = (n + 2 * kTile - 1) / (2 * kTile);
   volatile int* abort_flag = &sm.abort_flag;
   if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
   if (threadIdx.x == 0) {
-    mbar_init(&sm.q_full, 1);
     for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.q_full[i], 1);
+      mbar_init(&sm.q_empty[i], 1);
       mbar_init(&sm.k_full[i], 1);
-      mbar_init(&sm.k_empty[i], users);
+      mbar_init(&sm.k_empty[i], 2);
       mbar_init(&sm.v_full[i], 1);
-      mbar_init(&sm.v_empty[i], users);
+      mbar_init(&sm.v_empty[i], 2);
       mbar_init(&sm.o_done[i], 1);
       for (int bf = 0; bf < 2; ++bf) {
         mbar_init(&sm.s_full[i][bf], 1);
@@ -100,32 +113,41 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      mbar_expect_tx(&sm.q_full, users * kTileBytes);
-      for (int w = 0; w < users; ++w) {
-        tma_load_4d(sm.q[w], &map_q, &sm.q_full, 0, h, r0 + w * kTile, b);
-        tma_load_4d(sm.q[w] + kHalfBytes, &map_q, &sm.q_full, 64, h, r0 + w * kTile, b);
-      }
       bool ok = true;
-      for (int j = 0; j < nkt && ok; ++j) {
-        const int st = j & 1;
-        if (j >= 2) ok = mbar_wait(&sm.k_empty[st], ((j - 2) >> 1) & 1, abort_flag, a.status, code);
-        if (!ok) break;
-        mbar_expect_tx(&sm.k_full[st], kTileBytes);
-        tma_load_4d(sm.k[st], &map_k, &sm.k_full[st], 0, g, j * kTile, b);
-        tma_load_4d(sm.k[st] + kHalfBytes, &map_k, &sm.k_full[st], 64, g, j * kTile, b);
-        if (j >= 2) ok = mbar_wait(&sm.v_empty[st], ((j - 2) >> 1) & 1, abort_flag, a.status, code);
-        if (!ok) break;
-        mbar_expect_tx(&sm.v_full[st], kTileBytes);
-        tma_load_4d(sm.v[st], &map_v, &sm.v_full[st], 0, g, j * kTile, b);
-        tma_load_4d(sm.v[st] + kHalfBytes, &map_v, &sm.v_full[st], 64, g, j * kTile, b);
+      int kv = 0;                                      // K/V tiles loaded so far (stage = kv & 1)
+      int nq[2] = {0, 0};                              // Q loads issued per tile
+      for (int it = 0; it < nblk && ok; ++it) {
+        const Block bk = block_of(nblk - 1 - it, n);   // longest block first
+        for (int w = 0; w < 2 && ok; ++w) {
+          if (w == 1 && !bk.nkt1) break;
+          // the S MMAs of the previous block have finished reading this Q tile
+          if (nq[w] > 0) ok = mbar_wait(&sm.q_empty[w], (nq[w] - 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+          ++nq[w];
+          mbar_expect_tx(&sm.q_full[w], kTileBytes);
+          tma_load_4d(sm.q[w], &map_q, &sm.q_full[w], 0, h, bk.r0 + w * kTile, b);
+          tma_load_4d(sm.q[w] + kHalfBytes, &map_q, &sm.q_full[w], 64, h, bk.r0 + w * kTile, b);
+        }
+        for (int j = 0; j < bk.nkt && ok; ++j, ++kv) {
+          const int st = kv & 1;
+          if (kv >= 2) ok = mbar_wait(&sm.k_empty[st], ((kv - 2) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+          mbar_expect_tx(&sm.k_full[st], kTileBytes);
+          tma_load_4d(sm.k[st], &map_k, &sm.k_full[st], 0, g, j * kTile, b);
+          tma_load_4d(sm.k[st] + kHalfBytes, &map_k, &sm.k_full[st], 64, g, j * kTile, b);
+          if (kv >= 2) ok = mbar_wait(&sm.v_empty[st], ((kv - 2) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+          mbar_expect_tx(&sm.v_full[st], kTileBytes);
+          tma_load_4d(sm.v[st], &map_v, &sm.v_full[st], 0, g, j * kTile, b);
+          tma_load_4d(sm.v[st] + kHalfBytes, &map_v, &sm.v_full[st], 64, g, j * kTile, b);
+        }
       }
     }
     __syncwarp();
   } else if (warp >= kSoftmaxWarps) {
     // ---------------------------------------------------------------- MMA issue, one thread per tile
     const int w = warp - kSoftmaxWarps;
-    const int T = 2 * (w ? nkt1 : nkt0);           // half-steps of this tile
-    if (lane == 0 && T > 0) {
+    if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_bf16(kTile, kHalf, false, false);   // S = Q K^T (64 keys), both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
       // operand descriptors are built once; a k-step only adds a constant to the start-address field
@@ -135,40 +157,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
       const uint32_t t_base = tmem + w * 256, o_tmem = t_base + 128;
       bool ok = true;
-      // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
-      auto issue_s = [&](int t) {
-        const int j = t >> 1, st = j & 1, bf = t & 1;
-        if (bf == 0) {
-          ok = mbar_wait(&sm.k_full[st], (j >> 1) & 1, abort_flag, a.status, code);
-          if (!ok) return;
+      int kvu = 0;   // K/V tiles of the ring that earlier blocks used
+      int nq = 0;    // Q loads of this tile consumed
+      int hs = 0;    // half-steps of this tile done in earlier blocks (even)
+      for (int it = 0; it < nblk && ok; ++it) {
+        const Block bk = block_of(nblk - 1 - it, n);
+        const int nkt_w = w ? bk.nkt1 : bk.nkt0;
+        const int T = 2 * nkt_w;
+        // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
+        // landed (which also means the phase before it is closed), then release it
+        auto release = [&](int ring) {
+          const int st = ring & 1, par = (ring >> 1) & 1;
+          ok = mbar_wait(&sm.k_full[st], par, abort_flag, a.status, code);
+          if (ok) mbar_arrive(&sm.k_empty[st]);
+          if (ok) ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
+          if (ok) mbar_arrive(&sm.v_empty[st]);
+        };
+        // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
+        auto issue_s = [&](int t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) {
+            ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+            if (!ok) return;
+            tc_fence_after();
+          }
+          const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+            mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
+          }
+          mma_commit(&sm.s_full[w][bf]);
+          if (bf == 1) mma_commit(&sm.k_empty[st]);
+          if (t == T - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
+        };
+        if (T == 0) {
+          for (int j = 0; j < bk.nkt && ok; ++j) release(kvu + j);
+          kvu += bk.nkt;
+          continue;
+        }
+        ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
+        ++nq;
+        if (ok) issue_s(0);
+        if (ok) issue_s(1);
+        for (int t = 0; t < T && ok; ++t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+          if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
           tc_fence_after();
-        }
-        const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
+          const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-          mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
+          for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
+            mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+                   (t > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(&sm.o_done[w]);
+          if (bf == 1) mma_commit(&sm.v_empty[st]);
+          if (t + 2 < T) issue_s(t + 2);
         }
-        mma_commit(&sm.s_full[w][bf]);
-        if (bf == 1) mma_commit(&sm.k_empty[st]);
-      };
-      ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, code);
-      if (ok) issue_s(0);
-      if (ok) issue_s(1);
-      for (int t = 0; t < T && ok; ++t) {
-        const int j = t >> 1, st = j & 1, bf = t & 1;
-        if (bf == 0) ok = mbar_wait(&sm.v_full[st], (j >> 1) & 1, abort_flag, a.status, code);
-        if (ok) ok = mbar_wait(&sm.p_ready[w][bf], (t >> 1) & 1, abort_flag, a.status, code);
-        if (!ok) break;
-        tc_fence_after();
-        const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
-          mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
-                 (t > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(&sm.o_done[w]);
-        if (bf == 1) mma_commit(&sm.v_empty[st]);
-        if (t + 2 < T) issue_s(t + 2);
+        if (ok && nkt_w < bk.nkt) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
+        kvu += bk.nkt;
+        hs += T;
       }
     }
     __syncwarp();
@@ -176,85 +225,91 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---------------------------------------------------------------- softmax, thread = query row
     const int w = warp >> 2;
     const int row = threadIdx.x & (kTile - 1);
-    const int i = r0 + w * kTile + row;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t t_base = tmem + lane_base + w * 256;
     const uint32_t o_addr = t_base + 128;
-    const int T = 2 * (w ? nkt1 : nkt0);
     const float sc2 = a.scale * kLog2e;
-    float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int t = 0; t < T && ok; ++t) {
-      const int bf = t & 1;
-      const uint32_t s_addr = t_base + bf * kHalf;
-      ok = mbar_wait(&sm.s_full[w][bf], (t >> 1) & 1, abort_flag, a.status, code);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t s[64];
-      tmem_ld32(s_addr, s);
-      tmem_ld32(s_addr + 32, s + 32);
-      tmem_wait_ld();
-      if (t >= T - 2) {                 // inside the diagonal key tile: key 64 t + col is visible iff col <= lim
-        const int lim = i - t * kHalf;
-#pragma unroll
-        for (int col = 0; col < 64; ++col)
-          if (col > lim) s[col] = 0xff800000u;   // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-      for (int col = 0; col < 64; col += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
-      }
-      // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
-      const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
-      // A parity wait is only meaningful one phase behind the barrier, so o_done is followed on
-      // every half-step (PV(t-1) was issued a whole softmax ago: this wait is normally free).
-      if (t > 0) {
-        ok = mbar_wait(&sm.o_done[w], (t - 1) & 1, abort_flag, a.status, code);
+    int hs = 0;    // half-steps of this tile done in earlier blocks (even)
+    for (int it = 0; it < nblk && ok; ++it) {
+      const Block bk = block_of(nblk - 1 - it, n);
+      const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
+      if (T == 0) continue;
+      const int i = bk.r0 + w * kTile + row;             // query row of this thread
+      float m_used = -INFINITY, l = 0.f;
+      for (int t = 0; t < T && ok; ++t) {
+        const int bf = t & 1;
+        const uint32_t s_addr = t_base + bf * kHalf;
+        ok = mbar_wait(&sm.s_full[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
-      }
-      if (t > 0 && __any_sync(0xffffffffu, need)) {
-        // O holds every PV issued so far: it can be rescaled
         tc_fence_after();
-        const float f = need ? ex2(m_used - mx) : 1.f;
+        uint32_t s[64];
+        tmem_ld32(s_addr, s);
+        tmem_ld32(s_addr + 32, s + 32);
+        tmem_wait_ld();
+        if (t >= T - 2) {                 // inside the diagonal key tile: key 64 t + col is visible iff col <= lim
+          const int lim = i - t * kHalf;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t o[32];
-          tmem_ld32(o_addr + ch * 32, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int col = 0; col < 32; ++col) o[col] = __float_as_uint(__uint_as_float(o[col]) * f);
-          tmem_st32(o_addr + ch * 32, o);
+          for (int col = 0; col < 64; ++col)
+            if (col > lim) s[col] = 0xff800000u;   // -inf
         }
-        l *= f;
-      }
-      if (need) m_used = mx;
-      const float neg_m = -m_used;
-      float part[4] = {0.f, 0.f, 0.f, 0.f};
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t p[16];
-#pragma unroll
-        for (int c2 = 0; c2 < 16; ++c2) {
-          const float p0 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2]), sc2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2 + 1]), sc2, neg_m));
-          part[c2 & 1] += p0;
-          part[2 + (c2 & 1)] += p1;
-          p[c2] = pack_bf16(p0, p1);
+        for (int col = 0; col < 64; col += 8) {
+          mx0 = max3(mx0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
         }
-        tmem_st16(s_addr + ch * 16, p);
+        // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
+        const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
+        // A parity wait is only meaningful one phase behind the barrier, so o_done is followed on
+        // every half-step (PV(t-1) was issued a whole softmax ago: this wait is normally free).
+        if (t > 0) {
+          ok = mbar_wait(&sm.o_done[w], (hs + t - 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+        }
+        if (t > 0 && __any_sync(0xffffffffu, need)) {
+          // O holds every PV issued so far: it can be rescaled
+          tc_fence_after();
+          const float f = need ? ex2(m_used - mx) : 1.f;
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + ch * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int col = 0; col < 32; ++col) o[col] = __float_as_uint(__uint_as_float(o[col]) * f);
+            tmem_st32(o_addr + ch * 32, o);
+          }
+          l *= f;
+        }
+        if (need) m_used = mx;
+        const float neg_m = -m_used;
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t p[16];
+#pragma unroll
+          for (int c2 = 0; c2 < 16; ++c2) {
+            const float p0 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2]), sc2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2 + 1]), sc2, neg_m));
+            part[c2 & 1] += p0;
+            part[2 + (c2 & 1)] += p1;
+            p[c2] = pack_bf16(p0, p1);
+          }
+          tmem_st16(s_addr + ch * 16, p);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&sm.p_ready[w][bf]);
+        l += (part[0] + part[1]) + (part[2] + part[3]);
       }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&sm.p_ready[w][bf]);
-      l += (part[0] + part[1]) + (part[2] + part[3]);
-    }
-    if (ok && T > 0) ok = mbar_wait(&sm.o_done[w], (T - 1) & 1, abort_flag, a.status, code);
-    if (ok && T > 0) {
+      // epilogue of the block; the next block's first PV cannot start before these threads have
+      // delivered its P(0), i.e. after they are done reading O here
+      if (ok) ok = mbar_wait(&sm.o_done[w], (hs + T - 1) & 1, abort_flag, a.status, code);
+      if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
       __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.out) + b * a.osb + h * a.osh + (int64_t)i * a.osn;
@@ -276,6 +331,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
+      hs += T;
     }
   }
   tc_fence_before();
@@ -301,7 +357,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   const size_t smem = sizeof(AttnSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((a.n + 2 * kTile - 1) / (2 * kTile), a.Hq, a.B);
+  dim3 grid(a.Hq, a.B);
   attn_tc_kernel<<<grid, kThreads, smem, s>>>(mq, mk, mv, a);
   return cudaGetLastError();
 }

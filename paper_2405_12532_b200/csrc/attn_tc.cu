@@ -66,7 +66,7 @@ __device__ __forceinline__ Block block_of(int blk, int n) {
   return b;
 }
 
-__global__ void __maxnreg__(200)   // 10 warps x 200 registers fit the register file; launch bounds alone cap at 168
+__global__ void __maxnreg__(192)   // 10 warps x 192 registers fit the register file; launch bounds alone cap at 168
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrefillArgs a) {
   extern __shared__ uint8_t smem_raw[];

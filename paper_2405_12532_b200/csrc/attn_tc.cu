@@ -66,7 +66,8 @@ __device__ __forceinline__ Block block_of(int blk, int n) {
   return b;
 }
 
-__global__ void __maxnreg__(192)   // 10 warps x 192 registers fit the register file; launch bounds alone cap at 168
+// (10 warps put 3 on one scheduler partition: 16384 / (3 * 32) = 170 registers per thread at most)
+__global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrefillArgs a) {
   extern __shared__ uint8_t smem_raw[];

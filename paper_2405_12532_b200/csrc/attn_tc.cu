@@ -7,18 +7,18 @@
 // first MMAs and the output epilogue of consecutive blocks overlap instead of
 // paying a prologue per block, and every CTA of the grid does the same work.
 //   warps 0-3 / 4-7   softmax of tile 0 / 1, thread = one query row
-//   warp 8            MMA issue for both tiles (one lane)
-//   warp 9            TMA loads (one lane)
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each. S covers 128 keys
-// (one N = 128 MMA group, the shape that runs at full tensor rate); the softmax takes it as
-// two halves of 64 keys, writes each half's P (bf16) over S columns 0..31 / 32..63 and
-// signals it separately, so PV of the first half runs under the exponentials of the second.
-// The issuing thread alternates between the tiles:
-//     PVa0 PVb0 S0(j+1) | PVa1 PVb1 S1(j+1) | ...
-// so one tile's softmax (bound by the ex2 unit) overlaps the other tile's tensor work.
-// The running maximum used in the exponent is only raised when the row maximum has grown by
-// more than 2^8, which keeps rescaling of O (a TMEM round trip) rare; the final normalisation
-// uses the same maximum, so the result is the exact softmax.
+//   warp 8 / 9        MMA issue for tile 0 / 1 (one lane each)
+//   warp 10           TMA loads (one lane)
+// The keys are consumed in half-steps of 64. Tensor memory, per tile 256 of the
+// 512 columns: two S buffers of 64 fp32 columns and O (128 columns); P (bf16)
+// overwrites the first 32 columns of its S buffer. Because S is double
+// buffered, the issuing thread runs S(t+1) while the softmax of half-step t is
+// at work, and PV(t) follows as soon as P(t) is there:
+//     S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
+// The running maximum used in the exponent is only raised when the row maximum
+// has grown by more than 2^8, which keeps rescaling of O (a TMEM round trip)
+// rare; the final normalisation uses the same maximum, so the result is the
+// exact softmax.
 //
 // All mbarriers live across blocks, so every role counts the phases it has
 // consumed (a parity wait is only valid one phase behind the barrier).
@@ -39,7 +39,7 @@ constexpr int kHalf = 64;                   // keys per half-step
 constexpr int kHalfBytes = kTile * 128;     // one [128 rows x 64 bf16] swizzled half tile (half of D)
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128 x 128] bf16 tile = two halves along D
 constexpr int kSoftmaxWarps = 8;
-constexpr int kThreads = (kSoftmaxWarps + 2) * 32;
+constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
 constexpr float kRescaleStep = 8.0f;
 
 struct AttnSmem {
@@ -47,8 +47,8 @@ struct AttnSmem {
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
   uint64_t q_full[2], q_empty[2];                    // per tile
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage
-  uint64_t s_full[2], pa_ready[2], pb_ready[2], o_done[2];   // per tile; P of keys 0..63 / 64..127
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2];   // [tile][S buffer]
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -66,7 +66,6 @@ __device__ __forceinline__ Block block_of(int blk, int n) {
   return b;
 }
 
-// (10 warps put 3 on one scheduler partition: 16384 / (3 * 32) = 170 registers per thread at most)
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrefillArgs a) {
@@ -86,13 +85,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.q_full[i], 1);
       mbar_init(&sm.q_empty[i], 1);
       mbar_init(&sm.k_full[i], 1);
-      mbar_init(&sm.k_empty[i], 1);
+      mbar_init(&sm.k_empty[i], 2);
       mbar_init(&sm.v_full[i], 1);
-      mbar_init(&sm.v_empty[i], 1);
+      mbar_init(&sm.v_empty[i], 2);
       mbar_init(&sm.o_done[i], 1);
-      mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.pa_ready[i], kTile);
-      mbar_init(&sm.pb_ready[i], kTile);
+      for (int bf = 0; bf < 2; ++bf) {
+        mbar_init(&sm.s_full[i][bf], 1);
+        mbar_init(&sm.p_ready[i][bf], kTile);
+      }
     }
     sm.abort_flag = 0;
     fence_barrier_init();
@@ -107,7 +107,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t tmem = sm.tmem_base;
   const int code = PYR_ERR_TIMEOUT;
 
-  if (warp == kSoftmaxWarps + 1) {
+  if (warp == kSoftmaxWarps + 2) {
     // ---------------------------------------------------------------- TMA loads
     if (lane == 0) {
       prefetch_tensormap(&map_q);
@@ -144,89 +144,80 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == kSoftmaxWarps) {
-    // ---------------------------------------------------------------- MMA issue (one thread, both tiles)
+  } else if (warp >= kSoftmaxWarps) {
+    // ---------------------------------------------------------------- MMA issue, one thread per tile
+    const int w = warp - kSoftmaxWarps;
     if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // S = Q K^T, both K-major
+      constexpr uint32_t idesc_s = idesc_bf16(kTile, kHalf, false, false);   // S = Q K^T (64 keys), both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
       // operand descriptors are built once; a k-step only adds a constant to the start-address field
-      const uint64_t dq0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024), dq1 = smem_desc_sw128(smem_u32(sm.q[1]), 16, 1024);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[w]), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
       const uint64_t dv0 = smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
+      const uint32_t t_base = tmem + w * 256, o_tmem = t_base + 128;
       bool ok = true;
-      int kvu = 0;             // K/V tiles of the ring that earlier blocks used
-      int nq[2] = {0, 0};      // Q loads consumed per tile
-      int cnt[2] = {0, 0};     // key tiles done per tile in earlier blocks
+      int kvu = 0;   // K/V tiles of the ring that earlier blocks used
+      int nq = 0;    // Q loads of this tile consumed
+      int hs = 0;    // half-steps of this tile done in earlier blocks (even)
       for (int it = 0; it < nblk && ok; ++it) {
         const Block bk = block_of(nblk - 1 - it, n);
-        const int last_w = bk.nkt1 ? 1 : 0;
-        auto issue_s = [&](int w, int j, int st) {
-          const uint64_t qd = w ? dq1 : dq0, kd = st ? dk1 : dk0;
-          const uint32_t d_tmem = tmem + w * kTile;
+        const int nkt_w = w ? bk.nkt1 : bk.nkt0;
+        const int T = 2 * nkt_w;
+        // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
+        // landed (which also means the phase before it is closed), then release it
+        auto release = [&](int ring) {
+          const int st = ring & 1, par = (ring >> 1) & 1;
+          ok = mbar_wait(&sm.k_full[st], par, abort_flag, a.status, code);
+          if (ok) mbar_arrive(&sm.k_empty[st]);
+          if (ok) ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
+          if (ok) mbar_arrive(&sm.v_empty[st]);
+        };
+        // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
+        auto issue_s = [&](int t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) {
+            ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+            if (!ok) return;
+            tc_fence_after();
+          }
+          const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
             const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-            mma_ss(d_tmem, qd + off, kd + off, idesc_s, kk > 0);
+            mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
           }
-          mma_commit(&sm.s_full[w]);
-          if (j == (w ? bk.nkt1 : bk.nkt0) - 1) mma_commit(&sm.q_empty[w]);   // last read of this block's Q tile
+          mma_commit(&sm.s_full[w][bf]);
+          if (bf == 1) mma_commit(&sm.k_empty[st]);
+          if (t == T - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
         };
-        // PV over 64 keys: half 0 = P columns 0..31 and V rows 0..63, half 1 = the rest
-        auto issue_pv = [&](int w, int st, int half, bool accumulate) {
-          const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((half * kHalf * 128) >> 4);
-          const uint32_t d_tmem = tmem + (2 + w) * kTile, p_tmem = tmem + w * kTile + half * 32;
+        if (T == 0) {
+          for (int j = 0; j < bk.nkt && ok; ++j) release(kvu + j);
+          kvu += bk.nkt;
+          continue;
+        }
+        ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
+        ++nq;
+        if (ok) issue_s(0);
+        if (ok) issue_s(1);
+        for (int t = 0; t < T && ok; ++t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+          if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
-            mma_ts(d_tmem, p_tmem + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
+            mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+                   (t > 0 || kk > 0) ? 1u : 0u);
           mma_commit(&sm.o_done[w]);
-        };
-        for (int w = 0; w <= last_w && ok; ++w) {
-          ok = mbar_wait(&sm.q_full[w], nq[w] & 1, abort_flag, a.status, code);
-          ++nq[w];
+          if (bf == 1) mma_commit(&sm.v_empty[st]);
+          if (t + 2 < T) issue_s(t + 2);
         }
-        if (ok) ok = mbar_wait(&sm.k_full[kvu & 1], (kvu >> 1) & 1, abort_flag, a.status, code);
-        if (!ok) break;
-        tc_fence_after();
-        issue_s(0, 0, kvu & 1);
-        if (last_w) issue_s(1, 0, kvu & 1);
-        mma_commit(&sm.k_empty[kvu & 1]);
-        // Order per key tile j: PVa0 PVb0 S0(j+1) PVa1 PVb1 S1(j+1). While one tile's softmax runs,
-        // the other tile's groups keep the tensor pipe busy.
-        for (int j = 0; j < bk.nkt && ok; ++j) {
-          const int ring = kvu + j, st = ring & 1, st1 = (ring + 1) & 1;
-          ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
-          if (!ok) break;
-          bool k_next_ready = false;
-          for (int w = 0; w < 2 && ok; ++w) {
-            const int nkt_w = w ? bk.nkt1 : bk.nkt0;
-            if (j < nkt_w) {
-              const int par = (cnt[w] + j) & 1;
-              ok = mbar_wait(&sm.pa_ready[w], par, abort_flag, a.status, code);
-              if (!ok) break;
-              tc_fence_after();
-              issue_pv(w, st, 0, j > 0);
-              ok = mbar_wait(&sm.pb_ready[w], par, abort_flag, a.status, code);
-              if (!ok) break;
-              tc_fence_after();
-              issue_pv(w, st, 1, true);
-            }
-            if (w == last_w) mma_commit(&sm.v_empty[st]);
-            if (j + 1 < nkt_w) {
-              if (!k_next_ready) {
-                ok = mbar_wait(&sm.k_full[st1], ((ring + 1) >> 1) & 1, abort_flag, a.status, code);
-                if (!ok) break;
-                k_next_ready = true;
-                tc_fence_after();
-              }
-              issue_s(w, j + 1, st1);
-            }
-            if (w == last_w && j + 1 < bk.nkt) mma_commit(&sm.k_empty[st1]);
-          }
-        }
+        if (ok && nkt_w < bk.nkt) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
         kvu += bk.nkt;
-        cnt[0] += bk.nkt0;
-        cnt[1] += bk.nkt1;
+        hs += T;
       }
     }
     __syncwarp();
@@ -235,24 +226,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int w = warp >> 2;
     const int row = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + w * kTile;          // S (128 columns); P lands on columns 0..63
-    const uint32_t o_addr = tmem + lane_base + (2 + w) * kTile;
+    const uint32_t t_base = tmem + lane_base + w * 256;
+    const uint32_t o_addr = t_base + 128;
     const float sc2 = a.scale * kLog2e;
     bool ok = true;
-    int cnt = 0;    // key tiles of this tile done in earlier blocks
+    int hs = 0;    // half-steps of this tile done in earlier blocks (even)
     for (int it = 0; it < nblk && ok; ++it) {
       const Block bk = block_of(nblk - 1 - it, n);
-      const int nkt_w = w ? bk.nkt1 : bk.nkt0;
-      if (nkt_w == 0) continue;
+      const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
+      if (T == 0) continue;
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;
-      // one online-softmax step over 64 keys held in s[0..63]; P goes to 32 columns at p_addr.
-      // `od` = index of the o_done phase that must be complete before O may be rescaled.
-      auto half_step = [&](uint32_t* s, int lim, bool diag, bool first, uint32_t p_addr, int od, uint64_t* ready) {
-        if (diag) {
+      for (int t = 0; t < T && ok; ++t) {
+        const int bf = t & 1;
+        const uint32_t s_addr = t_base + bf * kHalf;
+        ok = mbar_wait(&sm.s_full[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t s[64];
+        tmem_ld32(s_addr, s);
+        tmem_ld32(s_addr + 32, s + 32);
+        tmem_wait_ld();
+        if (t >= T - 2) {                 // inside the diagonal key tile: key 64 t + col is visible iff col <= lim
+          const int lim = i - t * kHalf;
 #pragma unroll
           for (int col = 0; col < 64; ++col)
-            if (col > lim) s[col] = 0xff800000u;   // -inf: key not visible to this row
+            if (col > lim) s[col] = 0xff800000u;   // -inf
         }
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
@@ -262,15 +261,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
           mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
         }
-        // (-inf when every key of this half is hidden from the row: then nothing changes and P = 0)
+        // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
-        const bool need = mx > m_used + kRescaleStep;      // also true on the first half (m_used = -inf)
-        bool followed = false;
-        if (!first && __any_sync(0xffffffffu, need)) {
-          // O must hold every PV issued so far before it is rescaled
-          ok = mbar_wait(&sm.o_done[w], od & 1, abort_flag, a.status, code);
-          followed = true;
-          if (!ok) return;
+        const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
+        // A parity wait is only meaningful one phase behind the barrier, so o_done is followed on
+        // every half-step (PV(t-1) was issued a whole softmax ago: this wait is normally free).
+        if (t > 0) {
+          ok = mbar_wait(&sm.o_done[w], (hs + t - 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+        }
+        if (t > 0 && __any_sync(0xffffffffu, need)) {
+          // O holds every PV issued so far: it can be rescaled
           tc_fence_after();
           const float f = need ? ex2(m_used - mx) : 1.f;
 #pragma unroll
@@ -298,36 +299,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             part[2 + (c2 & 1)] += p1;
             p[c2] = pack_bf16(p0, p1);
           }
-          tmem_st16(p_addr + ch * 16, p);
+          tmem_st16(s_addr + ch * 16, p);
         }
-        l += (part[0] + part[1]) + (part[2] + part[3]);
-        // a parity wait is only valid one phase behind the barrier: follow o_done on every half
-        // (by now the PV in question was issued a whole half-step ago, so this is normally free)
-        if (!first && !followed) ok = mbar_wait(&sm.o_done[w], od & 1, abort_flag, a.status, code);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(ready);
-      };
-      for (int j = 0; j < nkt_w && ok; ++j) {
-        ok = mbar_wait(&sm.s_full[w], (cnt + j) & 1, abort_flag, a.status, code);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t sa[64], sb[64];
-        tmem_ld32(s_addr, sa);
-        tmem_ld32(s_addr + 32, sa + 32);
-        tmem_ld32(s_addr + 64, sb);
-        tmem_ld32(s_addr + 96, sb + 32);
-        tmem_wait_ld();
-        const bool diag = j == nkt_w - 1;          // key 128 j + col is visible iff col <= i - 128 j
-        const int lim = i - j * kTile;
-        const int od = 2 * (cnt + j);              // o_done phases: 2 j = PVa(j), 2 j + 1 = PVb(j)
-        half_step(sa, lim, diag, j == 0, s_addr, od - 1, &sm.pa_ready[w]);
-        if (!ok) break;
-        half_step(sb, lim - kHalf, diag, false, s_addr + 32, od, &sm.pb_ready[w]);
+        mbar_arrive(&sm.p_ready[w][bf]);
+        l += (part[0] + part[1]) + (part[2] + part[3]);
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
-      // delivered its P, i.e. after they are done reading O here
-      if (ok) ok = mbar_wait(&sm.o_done[w], (2 * (cnt + nkt_w) - 1) & 1, abort_flag, a.status, code);
+      // delivered its P(0), i.e. after they are done reading O here
+      if (ok) ok = mbar_wait(&sm.o_done[w], (hs + T - 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
@@ -350,7 +331,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
-      cnt += nkt_w;
+      hs += T;
     }
   }
   tc_fence_before();

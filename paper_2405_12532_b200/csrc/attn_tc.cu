@@ -49,6 +49,7 @@ struct AttnSmem {
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2];   // [tile][S buffer]
+  uint64_t turn[2][4];                               // [tile][warp of the tile]: that warp may run its exponentials
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -89,6 +90,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 2);
       mbar_init(&sm.o_done[i], 1);
+      for (int p = 0; p < 4; ++p) mbar_init(&sm.turn[i][p], 1);
       for (int bf = 0; bf < 2; ++bf) {
         mbar_init(&sm.s_full[i][bf], 1);
         mbar_init(&sm.p_ready[i][bf], kTile);
@@ -231,10 +233,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float sc2 = a.scale * kLog2e;
     bool ok = true;
     int hs = 0;    // half-steps of this tile done in earlier blocks (even)
+    // The two warps that share a scheduler (warp p of tile 0 and warp p of tile 1) take turns at the
+    // exponential loop, so that one tile's special-function work overlaps the other's TMEM loads,
+    // row maxima and barrier waits instead of both phases running in lockstep. Tile 0 goes first.
+    const int pair = warp & 3;
+    int turns = 0;  // turns taken so far (the same number on both tiles)
     for (int it = 0; it < nblk && ok; ++it) {
       const Block bk = block_of(nblk - 1 - it, n);
       const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
       if (T == 0) continue;
+      const int shared_steps = bk.nkt1 ? 2 * bk.nkt0 : 0;   // half-steps that both tiles have
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;
       for (int t = 0; t < T && ok; ++t) {
@@ -287,6 +295,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         if (need) m_used = mx;
         const float neg_m = -m_used;
+        const bool take_turn = t < shared_steps;
+        if (take_turn && (w == 1 || turns > 0)) {
+          ok = mbar_wait(&sm.turn[w][pair], (w ? turns : turns - 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+        }
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
@@ -300,6 +313,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             p[c2] = pack_bf16(p0, p1);
           }
           tmem_st16(s_addr + ch * 16, p);
+        }
+        if (take_turn) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.turn[w ^ 1][pair]);
+          ++turns;
         }
         tmem_wait_st();
         tc_fence_before();

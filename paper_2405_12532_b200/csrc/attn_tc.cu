@@ -48,7 +48,7 @@ struct AttnSmem {
   alignas(1024) uint8_t v[2][kTileBytes];
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
-  uint64_t s_full[2][2], p_ready[2][2], o_done[2];   // [tile][S buffer]
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
   uint64_t turn[2][4];                               // [tile][warp of the tile]: that warp may run its exponentials
   uint32_t tmem_base;
   int abort_flag;
@@ -89,11 +89,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.k_empty[i], 2);
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 2);
-      mbar_init(&sm.o_done[i], 1);
       for (int p = 0; p < 4; ++p) mbar_init(&sm.turn[i][p], 1);
       for (int bf = 0; bf < 2; ++bf) {
         mbar_init(&sm.s_full[i][bf], 1);
         mbar_init(&sm.p_ready[i][bf], kTile);
+        mbar_init(&sm.o_done[i][bf], 1);
       }
     }
     sm.abort_flag = 0;
@@ -213,7 +213,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
             mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
                    (t > 0 || kk > 0) ? 1u : 0u);
-          mma_commit(&sm.o_done[w]);
+          mma_commit(&sm.o_done[w][bf]);
           if (bf == 1) mma_commit(&sm.v_empty[st]);
           if (t + 2 < T) issue_s(t + 2);
         }
@@ -272,14 +272,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
         const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
-        // A parity wait is only meaningful one phase behind the barrier, so o_done is followed on
-        // every half-step (PV(t-1) was issued a whole softmax ago: this wait is normally free).
-        if (t > 0) {
-          ok = mbar_wait(&sm.o_done[w], (hs + t - 1) & 1, abort_flag, a.status, code);
-          if (!ok) break;
-        }
         if (t > 0 && __any_sync(0xffffffffu, need)) {
-          // O holds every PV issued so far: it can be rescaled
+          // O may be rescaled once it holds every PV up to PV(t-1), the last one these threads have
+          // fed (the pipe runs the MMAs in order). That PV is the next phase of o_done[(t-1) & 1]:
+          // the phase before it, PV(t-3), had finished before S(t-1) was produced, and the one after
+          // it needs P(t+1). So this parity wait is valid although the barrier is not followed.
+          ok = mbar_wait(&sm.o_done[w][(t - 1) & 1], ((hs + t - 1) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_used - mx) : 1.f;
 #pragma unroll
@@ -326,7 +325,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
       // delivered its P(0), i.e. after they are done reading O here
-      if (ok) ok = mbar_wait(&sm.o_done[w], (hs + T - 1) & 1, abort_flag, a.status, code);
+      if (ok) ok = mbar_wait(&sm.o_done[w][(T - 1) & 1], ((hs + T - 1) >> 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;

@@ -48,7 +48,7 @@ struct AttnSmem {
   alignas(1024) uint8_t v[2][kTileBytes];
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
-  uint64_t s_full[2], p_ready[2][2], o_done[2][2];   // per tile; [tile][half of the key tile]
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
   uint64_t turn[2][4];                               // [tile][warp of the tile]: that warp may run its exponentials
   uint32_t tmem_base;
   int abort_flag;
@@ -90,10 +90,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 2);
       for (int p = 0; p < 4; ++p) mbar_init(&sm.turn[i][p], 1);
-      mbar_init(&sm.s_full[i], 1);
-      for (int half = 0; half < 2; ++half) {
-        mbar_init(&sm.p_ready[i][half], kTile);
-        mbar_init(&sm.o_done[i][half], 1);
+      for (int bf = 0; bf < 2; ++bf) {
+        mbar_init(&sm.s_full[i][bf], 1);
+        mbar_init(&sm.p_ready[i][bf], kTile);
+        mbar_init(&sm.o_done[i][bf], 1);
       }
     }
     sm.abort_flag = 0;
@@ -150,21 +150,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---------------------------------------------------------------- MMA issue, one thread per tile
     const int w = warp - kSoftmaxWarps;
     if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // S = Q K^T (128 keys), both K-major
+      constexpr uint32_t idesc_s = idesc_bf16(kTile, kHalf, false, false);   // S = Q K^T (64 keys), both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
       // operand descriptors are built once; a k-step only adds a constant to the start-address field
       const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[w]), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
       const uint64_t dv0 = smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
-      const uint32_t s_tmem = tmem + w * 256, o_tmem = s_tmem + 128;
+      const uint32_t t_base = tmem + w * 256, o_tmem = t_base + 128;
       bool ok = true;
       int kvu = 0;   // K/V tiles of the ring that earlier blocks used
       int nq = 0;    // Q loads of this tile consumed
-      int cnt = 0;   // key tiles of this tile done in earlier blocks
+      int hs = 0;    // half-steps of this tile done in earlier blocks (even)
       for (int it = 0; it < nblk && ok; ++it) {
         const Block bk = block_of(nblk - 1 - it, n);
         const int nkt_w = w ? bk.nkt1 : bk.nkt0;
+        const int T = 2 * nkt_w;
         // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
         // landed (which also means the phase before it is closed), then release it
         auto release = [&](int ring) {
@@ -174,48 +175,51 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (ok) ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
           if (ok) mbar_arrive(&sm.v_empty[st]);
         };
-        if (nkt_w == 0) {
+        // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
+        auto issue_s = [&](int t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) {
+            ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+            if (!ok) return;
+            tc_fence_after();
+          }
+          const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+            mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
+          }
+          mma_commit(&sm.s_full[w][bf]);
+          if (bf == 1) mma_commit(&sm.k_empty[st]);
+          if (t == T - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
+        };
+        if (T == 0) {
           for (int j = 0; j < bk.nkt && ok; ++j) release(kvu + j);
           kvu += bk.nkt;
           continue;
         }
         ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
         ++nq;
-        for (int j = 0; j < nkt_w && ok; ++j) {
-          const int ring = kvu + j, st = ring & 1, par = (ring >> 1) & 1, ph = (cnt + j) & 1;
-          ok = mbar_wait(&sm.k_full[st], par, abort_flag, a.status, code);
+        if (ok) issue_s(0);
+        if (ok) issue_s(1);
+        for (int t = 0; t < T && ok; ++t) {
+          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+          if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
-          // S(j) lands on the columns that held S(j-1) and P(j-1): the pipe runs it after PV(j-1)
-          const uint64_t kd = st ? dk1 : dk0;
+          const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-            mma_ss(s_tmem, dq + off, kd + off, idesc_s, kk > 0);
-          }
-          mma_commit(&sm.s_full[w]);
-          mma_commit(&sm.k_empty[st]);
-          if (j == nkt_w - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
-          ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
-          const uint64_t vd = st ? dv1 : dv0;
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            // P of keys 64 half .. 64 half + 63: 32 columns of bf16 pairs, V rows 64 half ..
-            if (ok) ok = mbar_wait(&sm.p_ready[w][half], ph, abort_flag, a.status, code);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
-              mma_ts(o_tmem, s_tmem + half * 32 + kk * 8, vd + (uint64_t)((half * kHalf * 128 + kk * 2048) >> 4),
-                     idesc_o, (j > 0 || half > 0 || kk > 0) ? 1u : 0u);
-            mma_commit(&sm.o_done[w][half]);
-          }
-          if (!ok) break;
-          mma_commit(&sm.v_empty[st]);
+          for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
+            mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+                   (t > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(&sm.o_done[w][bf]);
+          if (bf == 1) mma_commit(&sm.v_empty[st]);
+          if (t + 2 < T) issue_s(t + 2);
         }
         if (ok && nkt_w < bk.nkt) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
         kvu += bk.nkt;
-        cnt += nkt_w;
+        hs += T;
       }
     }
     __syncwarp();
@@ -224,11 +228,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int w = warp >> 2;
     const int row = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_base = tmem + lane_base + w * 256;   // S: 128 fp32 columns; P(half) lands on columns 32 half ..
-    const uint32_t o_addr = s_base + 128;
+    const uint32_t t_base = tmem + lane_base + w * 256;
+    const uint32_t o_addr = t_base + 128;
     const float sc2 = a.scale * kLog2e;
     bool ok = true;
-    int cnt = 0;   // key tiles of this tile done in earlier blocks
+    int hs = 0;    // half-steps of this tile done in earlier blocks (even)
     // The two warps that share a scheduler (warp p of tile 0 and warp p of tile 1) take turns at the
     // exponential loop, so that one tile's special-function work overlaps the other's TMEM loads,
     // row maxima and barrier waits instead of both phases running in lockstep. Tile 0 goes first.
@@ -242,13 +246,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;
       for (int t = 0; t < T && ok; ++t) {
-        const int half = t & 1, ph = (cnt + (t >> 1)) & 1;
-        const uint32_t s_addr = s_base + half * kHalf;
-        if (half == 0) {
-          ok = mbar_wait(&sm.s_full[w], ph, abort_flag, a.status, code);
-          if (!ok) break;
-          tc_fence_after();
-        }
+        const int bf = t & 1;
+        const uint32_t s_addr = t_base + bf * kHalf;
+        ok = mbar_wait(&sm.s_full[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
+        if (!ok) break;
+        tc_fence_after();
         uint32_t s[64];
         tmem_ld32(s_addr, s);
         tmem_ld32(s_addr + 32, s + 32);
@@ -271,14 +273,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
         const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
         if (t > 0 && __any_sync(0xffffffffu, need)) {
-          // O may be rescaled once it holds every PV these threads have fed. On the first half of a
-          // key tile that is already so: S(j) was issued after PV(j-1) and the pipe runs in order.
-          // On the second half the PV of the first half may still be running; it is the next phase
-          // of o_done[0] (the one before it had finished before S(j) was produced).
-          if (half == 1) {
-            ok = mbar_wait(&sm.o_done[w][0], ph, abort_flag, a.status, code);
-            if (!ok) break;
-          }
+          // O may be rescaled once it holds every PV up to PV(t-1), the last one these threads have
+          // fed (the pipe runs the MMAs in order). That PV is the next phase of o_done[(t-1) & 1]:
+          // the phase before it, PV(t-3), had finished before S(t-1) was produced, and the one after
+          // it needs P(t+1). So this parity wait is valid although the barrier is not followed.
+          ok = mbar_wait(&sm.o_done[w][(t - 1) & 1], ((hs + t - 1) >> 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_used - mx) : 1.f;
 #pragma unroll
@@ -311,7 +311,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             part[2 + (c2 & 1)] += p1;
             p[c2] = pack_bf16(p0, p1);
           }
-          tmem_st16(s_base + half * 32 + ch * 16, p);
+          tmem_st16(s_addr + ch * 16, p);
         }
         if (take_turn) {
           __syncwarp();
@@ -320,12 +320,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&sm.p_ready[w][half]);
+        mbar_arrive(&sm.p_ready[w][bf]);
         l += (part[0] + part[1]) + (part[2] + part[3]);
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
       // delivered its P(0), i.e. after they are done reading O here
-      if (ok) ok = mbar_wait(&sm.o_done[w][1], (cnt + (T >> 1) - 1) & 1, abort_flag, a.status, code);
+      if (ok) ok = mbar_wait(&sm.o_done[w][(T - 1) & 1], ((hs + T - 1) >> 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
@@ -348,7 +348,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
-      cnt += T >> 1;
+      hs += T;
     }
   }
   tc_fence_before();

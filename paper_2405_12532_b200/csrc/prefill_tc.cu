@@ -2,12 +2,12 @@
 //
 // score_tc_kernel: Algorithm 1's "A_e <- weighted_avg(A[-L:, :-L], dim=-2)".
 // With the softmax statistics (lse) of the L recent queries known, a CTA owns
-// 128 context keys of one (sequence, selection group) and computes
-// S^T = K_tile . Q_tile^T on the tensor cores with the keys on the TMEM lane
-// axis. Each thread then owns one key and sums w_i * exp(s_ij - lse_i) over
-// the recent queries i of every head of the group, in a fixed order. The
-// L x c block of attention weights only ever exists as 128 x 128 tiles in
-// tensor memory.
+// one (sequence, head): its recent queries stay in shared memory and the
+// context keys stream through once. S^T = K_tile . Q_tile^T runs on the tensor
+// cores with the keys on the TMEM lane axis, so a thread owns one key and sums
+// w_i * exp(s_ij - lse_i) over the recent queries i. The L x c block of
+// attention weights only ever exists as 128 x 128 tiles in tensor memory.
+// score_reduce_kernel then adds the heads of a selection group in a fixed order.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -64,43 +64,53 @@ constexpr int kTileBytes = 2 * kHalfBytes; // a [128 x 128] bf16 tile = two halv
 enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 
 // ------------------------------------------------------------------ score kernel
-// Warps 0-3 and 4-7: two groups of 128 threads, thread = one key of the tile;
-// group w takes the steps s with s % 2 == w and TMEM buffer w. Warp 8: one
-// lane loads tiles by TMA and issues the MMAs.
+// A CTA owns one (sequence, head) and up to kMaxQTiles tiles of 128 recent
+// queries, which stay in shared memory while the context keys of the head
+// stream through once, 128 per tile. Per (key tile, query tile) step one lane
+// of warp 8 issues S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into
+// one of two TMEM buffers. Warps 0-3 take query columns 0..63 of the step,
+// warps 4-7 columns 64..127; a thread owns one key and sums
+// w_i * exp(s_ij - lse_i) over its columns of every query tile, then writes the
+// key's partial score of (head, query chunk, column half). A second kernel adds
+// the partial scores of a selection group in a fixed order.
 constexpr int kScoreThreads = 288;
+constexpr int kMaxQTiles = 4;              // query tiles resident per CTA
+constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
 
 struct ScoreSmem {
-  alignas(1024) uint8_t k[2][kTileBytes];
-  alignas(1024) uint8_t q[2][kTileBytes];
-  float bias[2][kTile];
-  double partial[kTile];
-  uint64_t ld_full[2], ld_empty[2], s_full[2], s_empty[2];
+  alignas(1024) uint8_t tiles[kScoreTiles][kTileBytes];
+  alignas(16) float bias[kMaxQTiles * kTile];
+  uint64_t q_full, k_full[kScoreTiles], k_empty[kScoreTiles], s_full[2], s_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 
 __global__ void __launch_bounds__(kScoreThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrefillArgs a) {
+score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrefillArgs a,
+                float* partial, int nchunk) {
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-  const int tile = blockIdx.x, gsel = blockIdx.y, b = blockIdx.z;
+  const int h = blockIdx.x, chunk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = a.n, L = a.L, c = n - L;
-  const int heads = a.Hq / a.G;
-  const int rep = a.Hq / a.Hkv;
-  const int nqt = (L + kTile - 1) / kTile;
-  const int steps = heads * nqt;
-  const int j0 = tile * kTile;
+  const int g = h / (a.Hq / a.Hkv);
+  const int q0 = chunk * kMaxQTiles * kTile;                        // first recent query of the chunk
+  const int nq = min(kMaxQTiles, (L - q0 + kTile - 1) / kTile);     // query tiles of this CTA (>= 1)
+  const int kst = kScoreTiles - nq;                                 // K stages (>= 2)
+  const int nkt = (c + kTile - 1) / kTile;
   volatile int* abort_flag = &sm.abort_flag;
   if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
   if (threadIdx.x == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int i = 0; i < kScoreTiles; ++i) {
+      mbar_init(&sm.k_full[i], 1);
+      mbar_init(&sm.k_empty[i], 1);
+    }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&sm.ld_full[i], 1);
-      mbar_init(&sm.ld_empty[i], 1);
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.s_empty[i], kTile);
+      mbar_init(&sm.s_empty[i], 2 * kTile);
     }
     sm.abort_flag = 0;
     fence_barrier_init();
@@ -119,87 +129,90 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
-      int g_prev = -1, kslot = 1;
-      // loads run one step ahead of the MMAs
-      auto issue_loads = [&](int s, int& g_prev_io, int& kslot_io) {
-        const int h = gsel * heads + s / nqt, qt = s % nqt, g = h / rep;
-        const int st = s & 1;
-        uint32_t bytes = kTileBytes;
-        if (g != g_prev_io) { kslot_io ^= 1; bytes += kTileBytes; }
-        mbar_expect_tx(&sm.ld_full[st], bytes);
-        if (g != g_prev_io) {
-          tma_load_4d(sm.k[kslot_io], &map_k, &sm.ld_full[st], 0, g, j0, b);
-          tma_load_4d(sm.k[kslot_io] + kHalfBytes, &map_k, &sm.ld_full[st], 64, g, j0, b);
-          g_prev_io = g;
-        }
-        tma_load_4d(sm.q[st], &map_q, &sm.ld_full[st], 0, h, c + qt * kTile, b);
-        tma_load_4d(sm.q[st] + kHalfBytes, &map_q, &sm.ld_full[st], 64, h, c + qt * kTile, b);
+      mbar_expect_tx(&sm.q_full, (uint32_t)nq * kTileBytes);
+      for (int qt = 0; qt < nq; ++qt) {
+        tma_load_4d(sm.tiles[qt], &map_q, &sm.q_full, 0, h, c + q0 + qt * kTile, b);
+        tma_load_4d(sm.tiles[qt] + kHalfBytes, &map_q, &sm.q_full, 64, h, c + q0 + qt * kTile, b);
+      }
+      auto load_k = [&](int j) {
+        const int st = j % kst;
+        uint8_t* dst = sm.tiles[nq + st];
+        mbar_expect_tx(&sm.k_full[st], kTileBytes);
+        tma_load_4d(dst, &map_k, &sm.k_full[st], 0, g, j * kTile, b);
+        tma_load_4d(dst + kHalfBytes, &map_k, &sm.k_full[st], 64, g, j * kTile, b);
       };
-      int kslot_of_step[2] = {0, 0};
-      issue_loads(0, g_prev, kslot);
-      kslot_of_step[0] = kslot;
-      bool ok = true;
-      for (int s = 0; s < steps && ok; ++s) {
-        const int st = s & 1;
-        if (s + 1 < steps) {
-          // the stage of step s+1 was read by the MMAs of step s-1
-          if (s >= 1) ok = mbar_wait(&sm.ld_empty[(s + 1) & 1], ((s - 1) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+      for (int j = 0; j < kst - 1 && j < nkt; ++j) load_k(j);
+      bool ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, kTimeoutScore);
+      int s = 0;   // step = (key tile, query tile)
+      for (int j = 0; j < nkt && ok; ++j) {
+        const int st = j % kst;
+        // keep kst - 1 key tiles in flight: tile j + kst - 1 goes to the stage tile j - 1 used
+        if (j + kst - 1 < nkt) {
+          if (j >= 1) ok = mbar_wait(&sm.k_empty[(j - 1) % kst], ((j - 1) / kst) & 1, abort_flag, a.status, kTimeoutScore);
           if (!ok) break;
-          issue_loads(s + 1, g_prev, kslot);
-          kslot_of_step[(s + 1) & 1] = kslot;
+          load_k(j + kst - 1);
         }
-        ok = mbar_wait(&sm.ld_full[st], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-        if (!ok) break;
-        if (s >= 2) ok = mbar_wait(&sm.s_empty[st], ((s - 2) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t ka = smem_u32(sm.k[kslot_of_step[st]]), qa = smem_u32(sm.q[st]);
-        const uint32_t d_tmem = tmem + st * kTile;
+        ok = mbar_wait(&sm.k_full[st], (j / kst) & 1, abort_flag, a.status, kTimeoutScore);
+        const uint32_t ka = smem_u32(sm.tiles[nq + st]);
+        for (int qt = 0; qt < nq && ok; ++qt, ++s) {
+          const int buf = s & 1;
+          if (s >= 2) ok = mbar_wait(&sm.s_empty[buf], ((s - 2) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t qa = smem_u32(sm.tiles[qt]);
+          const uint32_t d_tmem = tmem + buf * kTile;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          mma_ss(d_tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc, kk > 0);
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+            mma_ss(d_tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc, kk > 0);
+          }
+          mma_commit(&sm.s_full[buf]);
+          if (qt == nq - 1) mma_commit(&sm.k_empty[st]);
         }
-        mma_commit(&sm.s_full[st]);
-        mma_commit(&sm.ld_empty[st]);
       }
     }
     __syncwarp();
   } else {
-    const int wg = warp >> 2;                 // 0 or 1
+    const int wg = warp >> 2;                 // column half of every step
     const int key = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float sc2 = a.scale * kLog2e;
-    double total = 0.0;
-    bool ok = true;
-    for (int s = wg; s < steps && ok; s += 2) {
-      const int h = gsel * heads + s / nqt, qt = s % nqt;
-      const int i = qt * kTile + key;          // this thread prepares the bias of recent query i
-      // the bias buffer of this group is free: every thread passed the barrier below after its reads
-      sm.bias[wg][key] = i < L ? log2f(a.w[i]) - a.lse[((int64_t)b * a.Hq + h) * n + c + i] * kLog2e : -INFINITY;
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + wg), "r"(kTile) : "memory");
-      ok = mbar_wait(&sm.s_full[wg], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-      if (!ok) break;
-      tc_fence_after();
-      float part[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem + lane_base + wg * kTile + ch * 32, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int col = 0; col < 32; ++col)
-          part[col & 3] += ex2(fmaf(__uint_as_float(r[col]), sc2, sm.bias[wg][ch * 32 + col]));
-      }
-      tc_fence_before();
-      mbar_arrive(&sm.s_empty[wg]);
-      total += (double)((part[0] + part[1]) + (part[2] + part[3]));
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + wg), "r"(kTile) : "memory");
+    // bias of recent query i: log2 w_i - lse_i log2 e; -inf beyond the window (those Q rows are zero fill)
+    for (int i = threadIdx.x; i < nq * kTile; i += 2 * kTile) {
+      const int qi = q0 + i;
+      sm.bias[i] = qi < L ? log2f(a.w[qi]) - a.lse[((int64_t)b * a.Hq + h) * n + c + qi] * kLog2e : -INFINITY;
     }
-    if (wg == 1) sm.partial[key] = total;
-    asm volatile("bar.sync 3, 256;" ::: "memory");
-    if (wg == 0 && j0 + key < c && !*abort_flag)
-      a.score[((int64_t)b * a.G + gsel) * c + j0 + key] = (float)((total + sm.partial[key]) / (double)heads);
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    float* dst = partial + (((int64_t)b * a.Hq + h) * nchunk + chunk) * 2 * (int64_t)c + (int64_t)wg * c;
+    bool ok = true;
+    int s = 0;
+    for (int j = 0; j < nkt && ok; ++j) {
+      double total = 0.0;
+      for (int qt = 0; qt < nq && ok; ++qt, ++s) {
+        const int buf = s & 1;
+        ok = mbar_wait(&sm.s_full[buf], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t r[64];
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&sm.s_empty[buf]);          // the values are in registers: the buffer can be refilled
+        const float4* bias4 = reinterpret_cast<const float4*>(&sm.bias[qt * kTile + wg * 64]);
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c4 = 0; c4 < 16; ++c4) {
+          const float4 bv = bias4[c4];
+          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
+          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
+          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
+          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
+        }
+        total += (double)((part[0] + part[1]) + (part[2] + part[3]));
+      }
+      if (ok && j * kTile + key < c) dst[j * kTile + key] = (float)total;
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -209,6 +222,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   }
 }
 
+// score[b, g, j] = mean over the heads of group g of their summed partial scores, added in a fixed order.
+__global__ void score_reduce_kernel(const float* __restrict__ partial, float* __restrict__ score, int c, int G,
+                                    int rows_per_group, int heads, const int* status) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const int gsel = blockIdx.y, b = blockIdx.z;
+  if (j >= c || *status != 0) return;
+  const float* src = partial + ((int64_t)b * G + gsel) * rows_per_group * (int64_t)c + j;
+  double acc = 0.0;
+  for (int r = 0; r < rows_per_group; ++r) acc += (double)src[(int64_t)r * c];
+  score[((int64_t)b * G + gsel) * c + j] = (float)(acc / (double)heads);
+}
+
 }  // namespace
 
 bool score_tc_supported(const PrefillArgs& a) {
@@ -216,7 +241,9 @@ bool score_tc_supported(const PrefillArgs& a) {
 }
 bool tensor_maps_available() { return encode_fn() != nullptr; }
 
-cudaError_t launch_score_tc(const PrefillArgs& a, cudaStream_t s) {
+int score_tc_chunks(int L) { return ((L + kTile - 1) / kTile + kMaxQTiles - 1) / kMaxQTiles; }
+
+cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s) {
   const int c = a.n - a.L;
   if (c <= 0) return cudaSuccess;
   CUtensorMap mq, mk;
@@ -226,8 +253,14 @@ cudaError_t launch_score_tc(const PrefillArgs& a, cudaStream_t s) {
   const size_t smem = sizeof(ScoreSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((c + kTile - 1) / kTile, a.G, a.B);
-  score_tc_kernel<<<grid, kScoreThreads, smem, s>>>(mq, mk, a);
+  const int nchunk = score_tc_chunks(a.L);
+  dim3 grid(a.Hq, nchunk, a.B);
+  score_tc_kernel<<<grid, kScoreThreads, smem, s>>>(mq, mk, a, partial, nchunk);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int heads = a.Hq / a.G;
+  dim3 rgrid((c + 255) / 256, a.G, a.B);
+  score_reduce_kernel<<<rgrid, 256, 0, s>>>(partial, a.score, c, a.G, heads * nchunk * 2, heads, a.status);
   return cudaGetLastError();
 }
 

@@ -24,7 +24,7 @@ constexpr size_t kAlign = 256;
 std::atomic<uint64_t> g_launches{0};   // kernels launched by this process through the library
 
 struct Layout {
-  size_t status, w, score, lse, idx, pos0, pos1, part_acc, part_ml, total;
+  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, total;
   std::vector<LayerPlan> layers;
 };
 
@@ -68,6 +68,10 @@ void plan(const pyr_config_t* c, Layout* lay) {
   lay->status = off; off = align_up(off + pyr::kStatusWords * sizeof(int), kAlign);
   lay->w = off;      off = align_up(off + (size_t)L * 4, kAlign);
   lay->score = off;  off = align_up(off + B * G * (size_t)(c0 > 0 ? c0 : 1) * 4, kAlign);
+  // per-head partial scores of the tensor-core score kernel (bf16, head_dim 128 only)
+  lay->score_part = off;
+  if (c->dtype == PYR_BF16 && D == 128 && c0 > 0)
+    off = align_up(off + B * Hq * (size_t)pyr::score_tc_chunks(L) * 2 * (size_t)c0 * 4, kAlign);
   lay->lse = off;    off = align_up(off + B * Hq * (size_t)N * 4, kAlign);
   lay->idx = off;    off = align_up(off + B * G * (size_t)N * 4, kAlign);
   lay->pos0 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);
@@ -311,9 +315,9 @@ pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, con
   if (e != cudaSuccess) return PYR_ERR_CUDA;
   g_launches += 1;
   if (p.c > 0) {
-    e = tc_score ? pyr::launch_score_tc(a, s) : pyr::launch_score_simt(a, s);
+    e = tc_score ? pyr::launch_score_tc(a, at<float>(c, c->lay.score_part), s) : pyr::launch_score_simt(a, s);
     if (e != cudaSuccess) return PYR_ERR_CUDA;
-    g_launches += 1;
+    g_launches += tc_score ? 2 : 1;
   }
   c->phase = 1;
   c->last_prefilled = layer;

@@ -185,33 +185,59 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     asm volatile("bar.sync 1, 256;" ::: "memory");
     float* dst = partial + (((int64_t)b * a.Hq + h) * nchunk + chunk) * 2 * (int64_t)c + (int64_t)wg * c;
     bool ok = true;
-    int s = 0;
-    for (int j = 0; j < nkt && ok; ++j) {
-      double total = 0.0;
-      for (int qt = 0; qt < nq && ok; ++qt, ++s) {
-        const int buf = s & 1;
-        ok = mbar_wait(&sm.s_full[buf], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t r[64];
-        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
-        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&sm.s_empty[buf]);          // the values are in registers: the buffer can be refilled
-        const float4* bias4 = reinterpret_cast<const float4*>(&sm.bias[qt * kTile + wg * 64]);
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
+    const int steps = nkt * nq;
+    // The TMEM load of step s+1 is issued before the exponentials of step s, so that its latency
+    // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
+    uint32_t ra[64], rb[64];
+    auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
+      const int buf = s & 1;
+      ok = mbar_wait(&sm.s_full[buf], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+      if (!ok) return;
+      tc_fence_after();
+      tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
+      tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
+    };
+    auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&sm.s_empty[s & 1]);
+    };
+    auto weigh = [&](const uint32_t* r, int qt) -> float {
+      const float4* bias4 = reinterpret_cast<const float4*>(&sm.bias[qt * kTile + wg * 64]);
+      float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c4 = 0; c4 < 16; ++c4) {
-          const float4 bv = bias4[c4];
-          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
-          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
-          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
-          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
-        }
-        total += (double)((part[0] + part[1]) + (part[2] + part[3]));
+      for (int c4 = 0; c4 < 16; ++c4) {
+        const float4 bv = bias4[c4];
+        part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
+        part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
+        part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
+        part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
       }
-      if (ok && j * kTile + key < c) dst[j * kTile + key] = (float)total;
+      return (part[0] + part[1]) + (part[2] + part[3]);
+    };
+    double total = 0.0;
+    int j = 0, qt = 0;
+    auto account = [&](float v) {               // adds step (j, qt); after a key tile's last query tile, stores
+      total += (double)v;
+      if (++qt == nq) {
+        if (j * kTile + key < c) dst[j * kTile + key] = (float)total;
+        total = 0.0; qt = 0; ++j;
+      }
+    };
+    fetch(0, ra);
+    if (ok) landed(0);
+    for (int s = 0; s < steps && ok; s += 2) {
+      if (s + 1 < steps) fetch(s + 1, rb);
+      if (!ok) break;
+      const float va = weigh(ra, qt);
+      if (s + 1 < steps) landed(s + 1);
+      account(va);
+      if (s + 1 >= steps) break;
+      if (s + 2 < steps) fetch(s + 2, ra);
+      if (!ok) break;
+      const float vb = weigh(rb, qt);
+      if (s + 2 < steps) landed(s + 2);
+      account(vb);
     }
   }
   tc_fence_before();

@@ -64,46 +64,62 @@ constexpr int kTileBytes = 2 * kHalfBytes; // a [128 x 128] bf16 tile = two halv
 enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 
 // ------------------------------------------------------------------ score kernel
-// A CTA owns one (sequence, head) and up to kMaxQTiles tiles of 128 recent
+// Work item = one (sequence, head) and up to kMaxQTiles tiles of 128 recent
 // queries, which stay in shared memory while the context keys of the head
-// stream through once, 128 per tile. Per (key tile, query tile) step one lane
-// of warp 8 issues S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into
-// one of two TMEM buffers. Warps 0-3 take query columns 0..63 of the step,
-// warps 4-7 columns 64..127; a thread owns one key and sums
-// w_i * exp(s_ij - lse_i) over its columns of every query tile, then writes the
-// key's partial score of (head, query chunk, column half). A second kernel adds
-// the partial scores of a selection group in a fixed order.
+// stream through once, 128 per tile. The grid is one CTA per SM; a CTA takes
+// items blockIdx.x, blockIdx.x + gridDim.x, ... so the K ring keeps running
+// from one item into the next. Per (key tile, query tile) step one lane of
+// warp 8 issues S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one
+// of two TMEM buffers. Warps 0-3 take query columns 0..63 of the step, warps
+// 4-7 columns 64..127; a thread owns one key and sums w_i * exp(s_ij - lse_i)
+// over its columns of every query tile, then writes the key's partial score of
+// (head, query chunk, column half). A second kernel adds the partial scores of
+// a selection group in a fixed order.
 constexpr int kScoreThreads = 288;
-constexpr int kMaxQTiles = 4;              // query tiles resident per CTA
+constexpr int kMaxQTiles = 4;              // query tiles resident per item
 constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
 
 struct ScoreSmem {
   alignas(1024) uint8_t tiles[kScoreTiles][kTileBytes];
-  alignas(16) float bias[kMaxQTiles * kTile];
-  uint64_t q_full, k_full[kScoreTiles], k_empty[kScoreTiles], s_full[2], s_empty[2];
+  alignas(16) float bias[2][kMaxQTiles * kTile];     // of this item / of the next one
+  uint64_t q_full, q_empty, k_full[kScoreTiles], k_empty[kScoreTiles], s_full[2], s_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 
+struct ScoreItem {
+  int b, h, chunk, q0, nq;
+};
+
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, PrefillArgs a,
-                float* partial, int nchunk) {
+                float* partial, int nchunk, int nitems) {
   extern __shared__ uint8_t smem_raw[];
   ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-  const int h = blockIdx.x, chunk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = a.n, L = a.L, c = n - L;
-  const int g = h / (a.Hq / a.Hkv);
-  const int q0 = chunk * kMaxQTiles * kTile;                        // first recent query of the chunk
-  const int nq = min(kMaxQTiles, (L - q0 + kTile - 1) / kTile);     // query tiles of this CTA (>= 1)
-  const int kst = kScoreTiles - nq;                                 // K stages (>= 2)
+  const int rep = a.Hq / a.Hkv;
+  const int nq_max = min(kMaxQTiles, (L + kTile - 1) / kTile);
+  const int kst = kScoreTiles - nq_max;                             // K stages (>= 2)
   const int nkt = (c + kTile - 1) / kTile;
+  const int my_items = ((int)blockIdx.x < nitems) ? (nitems - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  auto item_of = [&](int k) {                                       // k-th item of this CTA; heads vary fastest
+    const int id = blockIdx.x + k * gridDim.x;
+    ScoreItem it;
+    it.h = id % a.Hq;
+    it.chunk = (id / a.Hq) % nchunk;
+    it.b = id / (a.Hq * nchunk);
+    it.q0 = it.chunk * kMaxQTiles * kTile;
+    it.nq = min(kMaxQTiles, (L - it.q0 + kTile - 1) / kTile);
+    return it;
+  };
   volatile int* abort_flag = &sm.abort_flag;
   if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
+    mbar_init(&sm.q_empty, 1);
     for (int i = 0; i < kScoreTiles; ++i) {
       mbar_init(&sm.k_full[i], 1);
       mbar_init(&sm.k_empty[i], 1);
@@ -125,49 +141,64 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const uint32_t tmem = sm.tmem_base;
 
   if (warp == 8) {
-    if (lane == 0) {
+    if (lane == 0 && my_items > 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
-      mbar_expect_tx(&sm.q_full, (uint32_t)nq * kTileBytes);
-      for (int qt = 0; qt < nq; ++qt) {
-        tma_load_4d(sm.tiles[qt], &map_q, &sm.q_full, 0, h, c + q0 + qt * kTile, b);
-        tma_load_4d(sm.tiles[qt] + kHalfBytes, &map_q, &sm.q_full, 64, h, c + q0 + qt * kTile, b);
-      }
-      auto load_k = [&](int j) {
-        const int st = j % kst;
-        uint8_t* dst = sm.tiles[nq + st];
-        mbar_expect_tx(&sm.k_full[st], kTileBytes);
-        tma_load_4d(dst, &map_k, &sm.k_full[st], 0, g, j * kTile, b);
-        tma_load_4d(dst + kHalfBytes, &map_k, &sm.k_full[st], 64, g, j * kTile, b);
-      };
-      for (int j = 0; j < kst - 1 && j < nkt; ++j) load_k(j);
-      bool ok = mbar_wait(&sm.q_full, 0, abort_flag, a.status, kTimeoutScore);
-      int s = 0;   // step = (key tile, query tile)
-      for (int j = 0; j < nkt && ok; ++j) {
-        const int st = j % kst;
-        // keep kst - 1 key tiles in flight: tile j + kst - 1 goes to the stage tile j - 1 used
-        if (j + kst - 1 < nkt) {
-          if (j >= 1) ok = mbar_wait(&sm.k_empty[(j - 1) % kst], ((j - 1) / kst) & 1, abort_flag, a.status, kTimeoutScore);
-          if (!ok) break;
-          load_k(j + kst - 1);
+      auto load_q = [&](const ScoreItem& it) {
+        mbar_expect_tx(&sm.q_full, (uint32_t)it.nq * kTileBytes);
+        for (int qt = 0; qt < it.nq; ++qt) {
+          tma_load_4d(sm.tiles[qt], &map_q, &sm.q_full, 0, it.h, c + it.q0 + qt * kTile, it.b);
+          tma_load_4d(sm.tiles[qt] + kHalfBytes, &map_q, &sm.q_full, 64, it.h, c + it.q0 + qt * kTile, it.b);
         }
-        ok = mbar_wait(&sm.k_full[st], (j / kst) & 1, abort_flag, a.status, kTimeoutScore);
-        const uint32_t ka = smem_u32(sm.tiles[nq + st]);
-        for (int qt = 0; qt < nq && ok; ++qt, ++s) {
-          const int buf = s & 1;
-          if (s >= 2) ok = mbar_wait(&sm.s_empty[buf], ((s - 2) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t qa = smem_u32(sm.tiles[qt]);
-          const uint32_t d_tmem = tmem + buf * kTile;
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            mma_ss(d_tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc, kk > 0);
+      };
+      const int total_kt = my_items * nkt;        // K tiles this CTA streams, numbered across its items
+      auto load_k = [&](int r) {
+        const ScoreItem it = item_of(r / nkt);
+        const int st = r % kst;
+        uint8_t* dst = sm.tiles[nq_max + st];
+        mbar_expect_tx(&sm.k_full[st], kTileBytes);
+        tma_load_4d(dst, &map_k, &sm.k_full[st], 0, it.h / rep, (r % nkt) * kTile, it.b);
+        tma_load_4d(dst + kHalfBytes, &map_k, &sm.k_full[st], 64, it.h / rep, (r % nkt) * kTile, it.b);
+      };
+      load_q(item_of(0));
+      for (int r = 0; r < kst - 1 && r < total_kt; ++r) load_k(r);
+      bool ok = true;
+      int s = 0;   // step = (key tile, query tile), numbered across items
+      for (int k = 0; k < my_items && ok; ++k) {
+        const ScoreItem it = item_of(k);
+        ok = mbar_wait(&sm.q_full, k & 1, abort_flag, a.status, kTimeoutScore);
+        for (int j = 0; j < nkt && ok; ++j) {
+          const int r = k * nkt + j, st = r % kst;
+          // keep kst - 1 key tiles in flight: tile r + kst - 1 goes to the stage tile r - 1 used
+          if (r + kst - 1 < total_kt) {
+            if (r >= 1) ok = mbar_wait(&sm.k_empty[(r - 1) % kst], ((r - 1) / kst) & 1, abort_flag, a.status, kTimeoutScore);
+            if (!ok) break;
+            load_k(r + kst - 1);
           }
-          mma_commit(&sm.s_full[buf]);
-          if (qt == nq - 1) mma_commit(&sm.k_empty[st]);
+          ok = mbar_wait(&sm.k_full[st], (r / kst) & 1, abort_flag, a.status, kTimeoutScore);
+          const uint32_t ka = smem_u32(sm.tiles[nq_max + st]);
+          for (int qt = 0; qt < it.nq && ok; ++qt, ++s) {
+            const int buf = s & 1;
+            if (s >= 2) ok = mbar_wait(&sm.s_empty[buf], ((s - 2) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t qa = smem_u32(sm.tiles[qt]);
+            const uint32_t d_tmem = tmem + buf * kTile;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+              mma_ss(d_tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc, kk > 0);
+            }
+            mma_commit(&sm.s_full[buf]);
+            if (qt == it.nq - 1) mma_commit(&sm.k_empty[st]);
+          }
+        }
+        if (ok && k + 1 < my_items) {
+          // the query tiles are free once this item's last MMAs have run
+          mma_commit(&sm.q_empty);
+          ok = mbar_wait(&sm.q_empty, k & 1, abort_flag, a.status, kTimeoutScore);
+          if (ok) load_q(item_of(k + 1));
         }
       }
     }
@@ -177,67 +208,91 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int key = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float sc2 = a.scale * kLog2e;
-    // bias of recent query i: log2 w_i - lse_i log2 e; -inf beyond the window (those Q rows are zero fill)
-    for (int i = threadIdx.x; i < nq * kTile; i += 2 * kTile) {
-      const int qi = q0 + i;
-      sm.bias[i] = qi < L ? log2f(a.w[qi]) - a.lse[((int64_t)b * a.Hq + h) * n + c + qi] * kLog2e : -INFINITY;
+    // bias of recent query i: log2 w_i - lse_i log2 e; -inf beyond the window (those Q rows are zero fill).
+    // A thread fetches its (at most two) entries of the next item while it works on this one.
+    auto bias_of = [&](const ScoreItem& it, int i) -> float {
+      const int qi = it.q0 + i;
+      return (i < it.nq * kTile && qi < L)
+                 ? log2f(a.w[qi]) - a.lse[((int64_t)it.b * a.Hq + it.h) * n + c + qi] * kLog2e
+                 : -INFINITY;
+    };
+    float nb0 = 0.f, nb1 = 0.f;
+    if (my_items > 0) {
+      const ScoreItem it = item_of(0);
+      nb0 = bias_of(it, threadIdx.x);
+      nb1 = bias_of(it, threadIdx.x + 2 * kTile);
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    float* dst = partial + (((int64_t)b * a.Hq + h) * nchunk + chunk) * 2 * (int64_t)c + (int64_t)wg * c;
     bool ok = true;
-    const int steps = nkt * nq;
-    // The TMEM load of step s+1 is issued before the exponentials of step s, so that its latency
-    // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
-    uint32_t ra[64], rb[64];
-    auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
-      const int buf = s & 1;
-      ok = mbar_wait(&sm.s_full[buf], (s >> 1) & 1, abort_flag, a.status, kTimeoutScore);
-      if (!ok) return;
-      tc_fence_after();
-      tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
-      tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
-    };
-    auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&sm.s_empty[s & 1]);
-    };
-    auto weigh = [&](const uint32_t* r, int qt) -> float {
-      const float4* bias4 = reinterpret_cast<const float4*>(&sm.bias[qt * kTile + wg * 64]);
-      float part[4] = {0.f, 0.f, 0.f, 0.f};
+    int sg = 0;   // steps of earlier items
+    for (int k = 0; k < my_items && ok; ++k) {
+      const ScoreItem it = item_of(k);
+      float* bias = sm.bias[k & 1];
+      bias[threadIdx.x] = nb0;
+      bias[threadIdx.x + 2 * kTile] = nb1;
+      // every thread is past its reads of this buffer (item k - 2) since it went through the barrier of item k - 1
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (k + 1 < my_items) {
+        const ScoreItem nx = item_of(k + 1);
+        nb0 = bias_of(nx, threadIdx.x);
+        nb1 = bias_of(nx, threadIdx.x + 2 * kTile);
+      }
+      float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * 2 * (int64_t)c + (int64_t)wg * c;
+      const int nq = it.nq;
+      const int steps = nkt * nq;
+      // The TMEM load of step s+1 is issued before the exponentials of step s, so that its latency
+      // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
+      uint32_t ra[64], rb[64];
+      auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
+        const int buf = (sg + s) & 1;
+        ok = mbar_wait(&sm.s_full[buf], ((sg + s) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+        if (!ok) return;
+        tc_fence_after();
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
+      };
+      auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&sm.s_empty[(sg + s) & 1]);
+      };
+      auto weigh = [&](const uint32_t* r, int qt) -> float {
+        const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 64]);
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c4 = 0; c4 < 16; ++c4) {
-        const float4 bv = bias4[c4];
-        part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
-        part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
-        part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
-        part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
+        for (int c4 = 0; c4 < 16; ++c4) {
+          const float4 bv = bias4[c4];
+          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
+          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
+          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
+          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
+        }
+        return (part[0] + part[1]) + (part[2] + part[3]);
+      };
+      double total = 0.0;
+      int j = 0, qt = 0;
+      auto account = [&](float v) {               // adds step (j, qt); after a key tile's last query tile, stores
+        total += (double)v;
+        if (++qt == nq) {
+          if (j * kTile + key < c) dst[j * kTile + key] = (float)total;
+          total = 0.0; qt = 0; ++j;
+        }
+      };
+      fetch(0, ra);
+      if (ok) landed(0);
+      for (int s = 0; s < steps && ok; s += 2) {
+        if (s + 1 < steps) fetch(s + 1, rb);
+        if (!ok) break;
+        const float va = weigh(ra, qt);
+        if (s + 1 < steps) landed(s + 1);
+        account(va);
+        if (s + 1 >= steps) break;
+        if (s + 2 < steps) fetch(s + 2, ra);
+        if (!ok) break;
+        const float vb = weigh(rb, qt);
+        if (s + 2 < steps) landed(s + 2);
+        account(vb);
       }
-      return (part[0] + part[1]) + (part[2] + part[3]);
-    };
-    double total = 0.0;
-    int j = 0, qt = 0;
-    auto account = [&](float v) {               // adds step (j, qt); after a key tile's last query tile, stores
-      total += (double)v;
-      if (++qt == nq) {
-        if (j * kTile + key < c) dst[j * kTile + key] = (float)total;
-        total = 0.0; qt = 0; ++j;
-      }
-    };
-    fetch(0, ra);
-    if (ok) landed(0);
-    for (int s = 0; s < steps && ok; s += 2) {
-      if (s + 1 < steps) fetch(s + 1, rb);
-      if (!ok) break;
-      const float va = weigh(ra, qt);
-      if (s + 1 < steps) landed(s + 1);
-      account(va);
-      if (s + 1 >= steps) break;
-      if (s + 2 < steps) fetch(s + 2, ra);
-      if (!ok) break;
-      const float vb = weigh(rb, qt);
-      if (s + 2 < steps) landed(s + 2);
-      account(vb);
+      sg += steps;
     }
   }
   tc_fence_before();
@@ -280,8 +335,12 @@ cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s
   cudaError_t e = cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int nchunk = score_tc_chunks(a.L);
-  dim3 grid(a.Hq, nchunk, a.B);
-  score_tc_kernel<<<grid, kScoreThreads, smem, s>>>(mq, mk, a, partial, nchunk);
+  const int nitems = a.B * nchunk * a.Hq;
+  int dev = 0, sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const int grid = nitems < sms ? nitems : sms;
+  score_tc_kernel<<<grid, kScoreThreads, smem, s>>>(mq, mk, a, partial, nchunk, nitems);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int heads = a.Hq / a.G;

@@ -68,21 +68,23 @@ enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 // queries, which stay in shared memory while the context keys of the head
 // stream through once, 128 per tile. The grid is one CTA per SM; a CTA takes
 // items blockIdx.x, blockIdx.x + gridDim.x, ... so the K ring keeps running
-// from one item into the next. Per (key tile, query tile) step one lane of
-// warp 8 issues S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one
-// of two TMEM buffers. Warps 0-3 take query columns 0..63 of the step, warps
+// from one item into the next: one lane of warp 9 issues the TMA loads. Per
+// (key tile, query tile) step one lane of warp 8 issues
+// S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one of four TMEM
+// buffers. Warps 0-3 take query columns 0..63 of the step, warps
 // 4-7 columns 64..127; a thread owns one key and sums w_i * exp(s_ij - lse_i)
 // over its columns of every query tile, then writes the key's partial score of
 // (head, query chunk, column half). A second kernel adds the partial scores of
 // a selection group in a fixed order.
-constexpr int kScoreThreads = 288;
+constexpr int kScoreThreads = 320;
+constexpr int kScoreBufs = 4;              // TMEM buffers of 128 columns
 constexpr int kMaxQTiles = 4;              // query tiles resident per item
 constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
 
 struct ScoreSmem {
   alignas(1024) uint8_t tiles[kScoreTiles][kTileBytes];
   alignas(16) float bias[2][kMaxQTiles * kTile];     // of this item / of the next one
-  uint64_t q_full, q_empty, k_full[kScoreTiles], k_empty[kScoreTiles], s_full[2], s_empty[2];
+  uint64_t q_full, q_empty, k_full[kScoreTiles], k_empty[kScoreTiles], s_full[kScoreBufs], s_empty[kScoreBufs];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -124,7 +126,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(&sm.k_full[i], 1);
       mbar_init(&sm.k_empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kScoreBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
       mbar_init(&sm.s_empty[i], 2 * kTile);
     }
@@ -132,7 +134,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     fence_barrier_init();
   }
   if (warp == 8) {
-    tmem_alloc(&sm.tmem_base, 256);
+    tmem_alloc(&sm.tmem_base, kScoreBufs * kTile);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -140,66 +142,69 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp == 8) {
+  if (warp == 9) {
+    // ---------------------------------------------------------------- TMA loads
     if (lane == 0 && my_items > 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
-      constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
-      auto load_q = [&](const ScoreItem& it) {
+      bool ok = true;
+      int r = 0;                                  // K tiles loaded so far, over all items of this CTA
+      int st = 0, use = 0;                        // stage of tile r and how often that stage was filled before
+      for (int k = 0; k < my_items && ok; ++k) {
+        const ScoreItem it = item_of(k);
+        // the query tiles are free once the previous item's last MMAs have run
+        if (k >= 1) ok = mbar_wait(&sm.q_empty, (k - 1) & 1, abort_flag, a.status, kTimeoutScore);
+        if (!ok) break;
         mbar_expect_tx(&sm.q_full, (uint32_t)it.nq * kTileBytes);
         for (int qt = 0; qt < it.nq; ++qt) {
           tma_load_4d(sm.tiles[qt], &map_q, &sm.q_full, 0, it.h, c + it.q0 + qt * kTile, it.b);
           tma_load_4d(sm.tiles[qt] + kHalfBytes, &map_q, &sm.q_full, 64, it.h, c + it.q0 + qt * kTile, it.b);
         }
-      };
-      const int total_kt = my_items * nkt;        // K tiles this CTA streams, numbered across its items
-      auto load_k = [&](int r) {
-        const ScoreItem it = item_of(r / nkt);
-        const int st = r % kst;
-        uint8_t* dst = sm.tiles[nq_max + st];
-        mbar_expect_tx(&sm.k_full[st], kTileBytes);
-        tma_load_4d(dst, &map_k, &sm.k_full[st], 0, it.h / rep, (r % nkt) * kTile, it.b);
-        tma_load_4d(dst + kHalfBytes, &map_k, &sm.k_full[st], 64, it.h / rep, (r % nkt) * kTile, it.b);
-      };
-      load_q(item_of(0));
-      for (int r = 0; r < kst - 1 && r < total_kt; ++r) load_k(r);
+        const int g = it.h / rep;
+        for (int j = 0; j < nkt && ok; ++j, ++r) {
+          if (use > 0) ok = mbar_wait(&sm.k_empty[st], (use - 1) & 1, abort_flag, a.status, kTimeoutScore);
+          if (!ok) break;
+          uint8_t* dst = sm.tiles[nq_max + st];
+          mbar_expect_tx(&sm.k_full[st], kTileBytes);
+          tma_load_4d(dst, &map_k, &sm.k_full[st], 0, g, j * kTile, it.b);
+          tma_load_4d(dst + kHalfBytes, &map_k, &sm.k_full[st], 64, g, j * kTile, it.b);
+          if (++st == kst) { st = 0; ++use; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 8) {
+    // ---------------------------------------------------------------- MMA issue
+    if (lane == 0 && my_items > 0) {
+      constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
       bool ok = true;
-      int s = 0;   // step = (key tile, query tile), numbered across items
+      int s = 0;                 // step = (key tile, query tile), numbered across items
+      int st = 0, use = 0;       // stage of the current K tile and how often it was filled before
       for (int k = 0; k < my_items && ok; ++k) {
         const ScoreItem it = item_of(k);
         ok = mbar_wait(&sm.q_full, k & 1, abort_flag, a.status, kTimeoutScore);
         for (int j = 0; j < nkt && ok; ++j) {
-          const int r = k * nkt + j, st = r % kst;
-          // keep kst - 1 key tiles in flight: tile r + kst - 1 goes to the stage tile r - 1 used
-          if (r + kst - 1 < total_kt) {
-            if (r >= 1) ok = mbar_wait(&sm.k_empty[(r - 1) % kst], ((r - 1) / kst) & 1, abort_flag, a.status, kTimeoutScore);
-            if (!ok) break;
-            load_k(r + kst - 1);
-          }
-          ok = mbar_wait(&sm.k_full[st], (r / kst) & 1, abort_flag, a.status, kTimeoutScore);
-          const uint32_t ka = smem_u32(sm.tiles[nq_max + st]);
+          ok = mbar_wait(&sm.k_full[st], use & 1, abort_flag, a.status, kTimeoutScore);
+          const uint64_t kd = smem_desc_sw128(smem_u32(sm.tiles[nq_max + st]), 16, 1024);
           for (int qt = 0; qt < it.nq && ok; ++qt, ++s) {
-            const int buf = s & 1;
-            if (s >= 2) ok = mbar_wait(&sm.s_empty[buf], ((s - 2) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+            const int buf = s & (kScoreBufs - 1);
+            if (s >= kScoreBufs)
+              ok = mbar_wait(&sm.s_empty[buf], ((s / kScoreBufs) - 1) & 1, abort_flag, a.status, kTimeoutScore);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t qa = smem_u32(sm.tiles[qt]);
+            const uint64_t qd = smem_desc_sw128(smem_u32(sm.tiles[qt]), 16, 1024);
             const uint32_t d_tmem = tmem + buf * kTile;
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-              mma_ss(d_tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc, kk > 0);
+              const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+              mma_ss(d_tmem, kd + off, qd + off, idesc, kk > 0);
             }
             mma_commit(&sm.s_full[buf]);
             if (qt == it.nq - 1) mma_commit(&sm.k_empty[st]);
           }
+          if (++st == kst) { st = 0; ++use; }
         }
-        if (ok && k + 1 < my_items) {
-          // the query tiles are free once this item's last MMAs have run
-          mma_commit(&sm.q_empty);
-          ok = mbar_wait(&sm.q_empty, k & 1, abort_flag, a.status, kTimeoutScore);
-          if (ok) load_q(item_of(k + 1));
-        }
+        if (ok) mma_commit(&sm.q_empty);
       }
     }
     __syncwarp();
@@ -243,8 +248,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
       uint32_t ra[64], rb[64];
       auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
-        const int buf = (sg + s) & 1;
-        ok = mbar_wait(&sm.s_full[buf], ((sg + s) >> 1) & 1, abort_flag, a.status, kTimeoutScore);
+        const int buf = (sg + s) & (kScoreBufs - 1);
+        ok = mbar_wait(&sm.s_full[buf], ((sg + s) / kScoreBufs) & 1, abort_flag, a.status, kTimeoutScore);
         if (!ok) return;
         tc_fence_after();
         tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
@@ -253,7 +258,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
         tmem_wait_ld();
         tc_fence_before();
-        mbar_arrive(&sm.s_empty[(sg + s) & 1]);
+        mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);
       };
       auto weigh = [&](const uint32_t* r, int qt) -> float {
         const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 64]);
@@ -299,7 +304,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   __syncthreads();
   if (warp == 8) {
     tc_fence_after();
-    tmem_dealloc(tmem, 256);
+    tmem_dealloc(tmem, kScoreBufs * kTile);
   }
 }
 

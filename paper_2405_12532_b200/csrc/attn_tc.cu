@@ -54,15 +54,24 @@ struct AttnSmem {
   int abort_flag;
 };
 
-// Geometry of one 256-row block of the head.
+// Geometry of one block of the head: two consecutive 128-row tiles that share their K/V tiles.
+// The tiles are paired from the last one down, so that with an odd number of tiles the block that
+// has a single tile is the one with the least work (the first 128 rows), not the one with the most.
 struct Block {
   int r0, nkt0, nkt1, nkt;   // first row; key tiles of tile 0 / tile 1 (0 = tile absent) / loaded
 };
 __device__ __forceinline__ Block block_of(int blk, int n) {
+  const int ntiles = (n + kTile - 1) / kTile;
   Block b;
-  b.r0 = blk * 2 * kTile;
-  b.nkt0 = 2 * blk + 1;                               // causal: the diagonal tile is the last one
-  b.nkt1 = (b.r0 + kTile < n) ? 2 * blk + 2 : 0;
+  if (ntiles & 1) {
+    b.r0 = blk ? (2 * blk - 1) * kTile : 0;
+    b.nkt0 = blk ? 2 * blk : 1;                         // causal: the diagonal tile is the last one
+    b.nkt1 = blk ? 2 * blk + 1 : 0;
+  } else {
+    b.r0 = blk * 2 * kTile;
+    b.nkt0 = 2 * blk + 1;
+    b.nkt1 = 2 * blk + 2;
+  }
   b.nkt = b.nkt1 ? b.nkt1 : b.nkt0;
   return b;
 }

@@ -46,6 +46,7 @@ struct AttnSmem {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
+  alignas(1024) uint8_t o_stage[2][kHalfBytes];      // per tile: [128 rows x 64 bf16] of O on its way out
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
@@ -78,7 +79,8 @@ __device__ __forceinline__ Block block_of(int blk, int n) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-               const __grid_constant__ CUtensorMap map_v, PrefillArgs a) {
+               const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+               PrefillArgs a) {
   extern __shared__ uint8_t smem_raw[];
   AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -337,28 +339,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (ok) ok = mbar_wait(&sm.o_done[w][(T - 1) & 1], ((hs + T - 1) >> 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
+      // O leaves through shared memory and a TMA store, 64 columns at a time (rows past n are
+      // clipped by the store). Thread 0 of the tile issues the stores and, before the staging
+      // buffer is written again, waits until they have read it.
       const float inv = 1.f / l;
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.out) + b * a.osb + h * a.osh + (int64_t)i * a.osn;
+      uint8_t* stage = sm.o_stage[w];
+      uint8_t* my_row = stage + row * 128;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t o[32];
-        tmem_ld32(o_addr + ch * 32, o);
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t o[64];
+        tmem_ld32(o_addr + hf * 64, o);
+        tmem_ld32(o_addr + hf * 64 + 32, o + 32);
         tmem_wait_ld();
-        if (i < n) {
+        if (row == 0) bulk_wait_read_all();
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(o[q4 * 8 + 0]) * inv, __uint_as_float(o[q4 * 8 + 1]) * inv);
-            pk.y = pack_bf16(__uint_as_float(o[q4 * 8 + 2]) * inv, __uint_as_float(o[q4 * 8 + 3]) * inv);
-            pk.z = pack_bf16(__uint_as_float(o[q4 * 8 + 4]) * inv, __uint_as_float(o[q4 * 8 + 5]) * inv);
-            pk.w = pack_bf16(__uint_as_float(o[q4 * 8 + 6]) * inv, __uint_as_float(o[q4 * 8 + 7]) * inv);
-            *reinterpret_cast<uint4*>(out + ch * 32 + q4 * 8) = pk;
-          }
+        for (int ch = 0; ch < 8; ++ch) {     // 16-byte chunk ch of the row sits at ch ^ (row & 7): the 128-byte swizzle
+          uint4 pk;
+          pk.x = pack_bf16(__uint_as_float(o[ch * 8 + 0]) * inv, __uint_as_float(o[ch * 8 + 1]) * inv);
+          pk.y = pack_bf16(__uint_as_float(o[ch * 8 + 2]) * inv, __uint_as_float(o[ch * 8 + 3]) * inv);
+          pk.z = pack_bf16(__uint_as_float(o[ch * 8 + 4]) * inv, __uint_as_float(o[ch * 8 + 5]) * inv);
+          pk.w = pack_bf16(__uint_as_float(o[ch * 8 + 6]) * inv, __uint_as_float(o[ch * 8 + 7]) * inv);
+          *reinterpret_cast<uint4*>(my_row + ((ch ^ (row & 7)) << 4)) = pk;
+        }
+        fence_proxy_async();
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
+        if (row == 0) {
+          tma_store_4d(&map_o, stage, hf * 64, h, bk.r0 + w * kTile, b);
+          bulk_commit();
         }
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
       hs += T;
     }
+    if (row == 0) bulk_wait_all();   // the last stores have left shared memory and are complete
   }
   tc_fence_before();
   __syncthreads();
@@ -375,8 +389,9 @@ bool prefill_tc_supported(const PrefillArgs& a) {
 }
 
 cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
-  CUtensorMap mq, mk, mv;
-  if (!make_tensor_map_bf16(&mq, a.q, a.B, a.n, a.Hq, a.D, a.qsb, a.qsn, a.qsh, kTile) ||
+  CUtensorMap mq, mk, mv, mo;
+  if (!make_tensor_map_bf16(&mo, a.out, a.B, a.n, a.Hq, a.D, a.osb, a.osn, a.osh, kTile) ||
+      !make_tensor_map_bf16(&mq, a.q, a.B, a.n, a.Hq, a.D, a.qsb, a.qsn, a.qsh, kTile) ||
       !make_tensor_map_bf16(&mk, a.k, a.B, a.n, a.Hkv, a.D, a.ksb, a.ksn, a.ksh, kTile) ||
       !make_tensor_map_bf16(&mv, a.v, a.B, a.n, a.Hkv, a.D, a.ksb, a.ksn, a.ksh, kTile))
     return cudaErrorInvalidValue;
@@ -384,7 +399,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(a.Hq, a.B);
-  attn_tc_kernel<<<grid, kThreads, smem, s>>>(mq, mk, mv, a);
+  attn_tc_kernel<<<grid, kThreads, smem, s>>>(mq, mk, mv, mo, a);
   return cudaGetLastError();
 }
 

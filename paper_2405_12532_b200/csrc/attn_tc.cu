@@ -46,10 +46,11 @@ struct AttnSmem {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
-  alignas(1024) uint8_t o_stage[2][kHalfBytes];      // per tile: [128 rows x 64 bf16] of O on its way out
+  alignas(1024) uint8_t o_stage[kTileBytes];         // a [128 x 128] bf16 tile of O on its way out (both tiles use it)
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
+  uint64_t stage_free;                               // the stores of one epilogue have read o_stage
   uint64_t turn[2][4];                               // [tile][warp of the tile]: that warp may run its exponentials
   uint32_t tmem_base;
   int abort_flag;
@@ -107,6 +108,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mbar_init(&sm.o_done[i][bf], 1);
       }
     }
+    mbar_init(&sm.stage_free, 1);
     sm.abort_flag = 0;
     fence_barrier_init();
   }
@@ -249,10 +251,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // row maxima and barrier waits instead of both phases running in lockstep. Tile 0 goes first.
     const int pair = warp & 3;
     int turns = 0;  // turns taken so far (the same number on both tiles)
+    // Epilogues use the staging tile in a fixed order: per block tile 0, then tile 1.
+    int ep_base = 0;             // epilogues of earlier blocks
+    bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
     for (int it = 0; it < nblk && ok; ++it) {
       const Block bk = block_of(nblk - 1 - it, n);
       const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
-      if (T == 0) continue;
+      if (T == 0) {
+        ep_base += 1;
+        continue;
+      }
       const int shared_steps = bk.nkt1 ? 2 * bk.nkt0 : 0;   // half-steps that both tiles have
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;
@@ -333,26 +341,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         tc_fence_before();
         mbar_arrive(&sm.p_ready[w][bf]);
         l += (part[0] + part[1]) + (part[2] + part[3]);
+        if (release_due) {       // only ever set in thread 0 of the tile
+          bulk_wait_read_all();
+          mbar_arrive(&sm.stage_free);
+          release_due = false;
+        }
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
       // delivered its P(0), i.e. after they are done reading O here
       if (ok) ok = mbar_wait(&sm.o_done[w][(T - 1) & 1], ((hs + T - 1) >> 1) & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
-      // O leaves through shared memory and a TMA store, 64 columns at a time (rows past n are
-      // clipped by the store). Thread 0 of the tile issues the stores and, before the staging
-      // buffer is written again, waits until they have read it.
+      // O leaves through shared memory and two TMA stores (rows past n are clipped by the store).
+      // The epilogue before this one (the other tile's, or this tile's of the previous block when
+      // that block had one tile) must have been read out of the staging tile first.
       const float inv = 1.f / l;
-      uint8_t* stage = sm.o_stage[w];
-      uint8_t* my_row = stage + row * 128;
+      const int seq = ep_base + w;
+      if (seq > 0) {
+        ok = mbar_wait(&sm.stage_free, (seq - 1) & 1, abort_flag, a.status, code);
+        if (!ok) break;
+      }
+      uint8_t* my_row = sm.o_stage + row * 128;
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         uint32_t o[64];
         tmem_ld32(o_addr + hf * 64, o);
         tmem_ld32(o_addr + hf * 64 + 32, o + 32);
         tmem_wait_ld();
-        if (row == 0) bulk_wait_read_all();
-        asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {     // 16-byte chunk ch of the row sits at ch ^ (row & 7): the 128-byte swizzle
           uint4 pk;
@@ -360,17 +375,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           pk.y = pack_bf16(__uint_as_float(o[ch * 8 + 2]) * inv, __uint_as_float(o[ch * 8 + 3]) * inv);
           pk.z = pack_bf16(__uint_as_float(o[ch * 8 + 4]) * inv, __uint_as_float(o[ch * 8 + 5]) * inv);
           pk.w = pack_bf16(__uint_as_float(o[ch * 8 + 6]) * inv, __uint_as_float(o[ch * 8 + 7]) * inv);
-          *reinterpret_cast<uint4*>(my_row + ((ch ^ (row & 7)) << 4)) = pk;
+          *reinterpret_cast<uint4*>(my_row + hf * kHalfBytes + ((ch ^ (row & 7)) << 4)) = pk;
         }
-        fence_proxy_async();
-        asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
-        if (row == 0) {
-          tma_store_4d(&map_o, stage, hf * 64, h, bk.r0 + w * kTile, b);
-          bulk_commit();
-        }
+      }
+      fence_proxy_async();
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
+      if (row == 0) {
+        tma_store_4d(&map_o, sm.o_stage, 0, h, bk.r0 + w * kTile, b);
+        tma_store_4d(&map_o, sm.o_stage + kHalfBytes, 64, h, bk.r0 + w * kTile, b);
+        bulk_commit();
+        release_due = true;   // signalled a little later, off the path to the next block's first P
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
       hs += T;
+      ep_base += bk.nkt1 ? 2 : 1;
+    }
+    if (release_due) {
+      bulk_wait_read_all();
+      mbar_arrive(&sm.stage_free);
     }
     if (row == 0) bulk_wait_all();   // the last stores have left shared memory and are complete
   }

@@ -355,6 +355,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // O leaves through shared memory and two TMA stores (rows past n are clipped by the store).
       // The epilogue before this one (the other tile's, or this tile's of the previous block when
       // that block had one tile) must have been read out of the staging tile first.
+      if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
       const float inv = 1.f / l;
       const int seq = ep_base + w;
       if (seq > 0) {
@@ -384,9 +385,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         tma_store_4d(&map_o, sm.o_stage, 0, h, bk.r0 + w * kTile, b);
         tma_store_4d(&map_o, sm.o_stage + kHalfBytes, 64, h, bk.r0 + w * kTile, b);
         bulk_commit();
-        release_due = true;   // signalled a little later, off the path to the next block's first P
+        if (w == 0) {         // tile 0 runs ahead of tile 1 and would wait for its next K tile anyway
+          bulk_wait_read_all();
+          mbar_arrive(&sm.stage_free);
+        } else {
+          release_due = true; // signalled a little later, off the path to the next block's first P
+        }
       }
-      if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
       hs += T;
       ep_base += bk.nkt1 ? 2 : 1;
     }

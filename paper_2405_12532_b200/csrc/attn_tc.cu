@@ -226,7 +226,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
             mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
                    (t > 0 || kk > 0) ? 1u : 0u);
-          mma_commit(&sm.o_done[w][bf]);
+          if (t >= T - 2) mma_commit(&sm.o_done[w][bf]);   // the block's last two PVs: one phase per block each
           if (bf == 1) mma_commit(&sm.v_empty[st]);
           if (t + 2 < T) issue_s(t + 2);
         }
@@ -252,6 +252,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int pair = warp & 3;
     int turns = 0;  // turns taken so far (the same number on both tiles)
     // Epilogues use the staging tile in a fixed order: per block tile 0, then tile 1.
+    int nb = 0;                  // blocks this tile has finished
     int ep_base = 0;             // epilogues of earlier blocks
     bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
     for (int it = 0; it < nblk && ok; ++it) {
@@ -293,10 +294,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
         if (t > 0 && __any_sync(0xffffffffu, need)) {
           // O may be rescaled once it holds every PV up to PV(t-1), the last one these threads have
-          // fed (the pipe runs the MMAs in order). That PV is the next phase of o_done[(t-1) & 1]:
-          // the phase before it, PV(t-3), had finished before S(t-1) was produced, and the one after
-          // it needs P(t+1). So this parity wait is valid although the barrier is not followed.
-          ok = mbar_wait(&sm.o_done[w][(t - 1) & 1], ((hs + t - 1) >> 1) & 1, abort_flag, a.status, code);
+          // fed. The issuing thread runs S(t+1) right after PV(t-1) and the pipe keeps that order,
+          // so S(t+1) having landed is the signal (its barrier is one phase ahead of what this
+          // thread has consumed, so the parity wait is valid); the block's last PVs have their own.
+          if (t + 1 < T) ok = mbar_wait(&sm.s_full[w][(t + 1) & 1], ((hs + t + 1) >> 1) & 1, abort_flag, a.status, code);
+          else ok = mbar_wait(&sm.o_done[w][0], nb & 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_used - mx) : 1.f;
@@ -349,7 +351,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
       // delivered its P(0), i.e. after they are done reading O here
-      if (ok) ok = mbar_wait(&sm.o_done[w][(T - 1) & 1], ((hs + T - 1) >> 1) & 1, abort_flag, a.status, code);
+      if (ok) ok = mbar_wait(&sm.o_done[w][1], nb & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
       // O leaves through shared memory and two TMA stores (rows past n are clipped by the store).
@@ -393,6 +395,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       hs += T;
+      ++nb;
       ep_base += bk.nkt1 ? 2 : 1;
     }
     if (release_due) {

@@ -143,7 +143,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tma_load_4d(sm.q[w], &map_q, &sm.q_full[w], 0, h, bk.r0 + w * kTile, b);
           tma_load_4d(sm.q[w] + kHalfBytes, &map_q, &sm.q_full[w], 64, h, bk.r0 + w * kTile, b);
         }
-        for (int j = 0; j < bk.nkt && ok; ++j, ++kv) {
+        // Key tiles go up in even blocks and down in odd ones: the tiles a block read last are the
+        // first ones the next block reads, so they are still in L2 (always going up evicts them all).
+        const bool down = it & 1;
+        for (int jj = 0; jj < bk.nkt && ok; ++jj, ++kv) {
+          const int j = down ? bk.nkt - 1 - jj : jj;
           const int st = kv & 1;
           if (kv >= 2) ok = mbar_wait(&sm.k_empty[st], ((kv - 2) >> 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
@@ -179,6 +183,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const Block bk = block_of(nblk - 1 - it, n);
         const int nkt_w = w ? bk.nkt1 : bk.nkt0;
         const int T = 2 * nkt_w;
+        // when the key tiles come in descending order, the one tile 0 does not read comes first
+        const int skip = ((it & 1) && nkt_w && nkt_w < bk.nkt) ? 1 : 0;
         // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
         // landed (which also means the phase before it is closed), then release it
         auto release = [&](int ring) {
@@ -190,7 +196,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         };
         // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
         auto issue_s = [&](int t) {
-          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          const int ring = kvu + skip + (t >> 1), st = ring & 1, bf = t & 1;
           if (bf == 0) {
             ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
             if (!ok) return;
@@ -211,12 +217,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           kvu += bk.nkt;
           continue;
         }
-        ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
+        if (skip) release(kvu);
+        if (ok) ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
         ++nq;
         if (ok) issue_s(0);
         if (ok) issue_s(1);
         for (int t = 0; t < T && ok; ++t) {
-          const int ring = kvu + (t >> 1), st = ring & 1, bf = t & 1;
+          const int ring = kvu + skip + (t >> 1), st = ring & 1, bf = t & 1;
           if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
           if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
@@ -230,7 +237,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (bf == 1) mma_commit(&sm.v_empty[st]);
           if (t + 2 < T) issue_s(t + 2);
         }
-        if (ok && nkt_w < bk.nkt) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
+        if (ok && nkt_w < bk.nkt && !skip) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
         kvu += bk.nkt;
         hs += T;
       }
@@ -275,8 +282,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         tmem_ld32(s_addr, s);
         tmem_ld32(s_addr + 32, s + 32);
         tmem_wait_ld();
-        if (t >= T - 2) {                 // inside the diagonal key tile: key 64 t + col is visible iff col <= lim
-          const int lim = i - t * kHalf;
+        // key tile of this half-step: they come in ascending order in even blocks, descending in odd ones
+        const int kt = (it & 1) ? (T >> 1) - 1 - (t >> 1) : (t >> 1);
+        if (kt == (T >> 1) - 1) {         // inside the diagonal key tile: key 128 kt + 64 (t & 1) + col is visible iff col <= lim
+          const int lim = i - (kt * kTile + (t & 1) * kHalf);
 #pragma unroll
           for (int col = 0; col < 64; ++col)
             if (col > lim) s[col] = 0xff800000u;   // -inf

@@ -269,7 +269,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
           part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
           part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
-          part[3] += ex2_fma(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));   // a quarter of the work off the MUFU
+          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
         }
         return (part[0] + part[1]) + (part[2] + part[3]);
       };

@@ -226,22 +226,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 2^x on the FMA and integer pipes instead of the special-function unit, for x <= 0 or so (results
-// below 2^-125 come out as 2^-125): round x to the nearest integer n with the 1.5 * 2^23 trick,
-// evaluate a degree-5 polynomial for 2^r on r = x - n in [-0.5, 0.5] (Chebyshev interpolation;
-// relative error 2.4e-7 in fp32), and add n to the exponent field.
-__device__ __forceinline__ float ex2_fma(float x) {
-  x = fmaxf(x, -125.0f);
-  const float t = x + 12582912.0f;
-  const float r = x - (t - 12582912.0f);
-  float p = 0.0013390863314270973f;
-  p = fmaf(p, r, 0.009676031768321991f);
-  p = fmaf(p, r, 0.055503569543361664f);
-  p = fmaf(p, r, 0.2402210682630539f);
-  p = fmaf(p, r, 0.6931471824645996f);
-  p = fmaf(p, r, 1.0000001192092896f);
-  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));

@@ -51,7 +51,6 @@ struct AttnSmem {
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
   uint64_t stage_free;                               // the stores of one epilogue have read o_stage
-  uint64_t turn[2][4];                               // [tile][warp of the tile]: that warp may run its exponentials
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -101,7 +100,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.k_empty[i], 2);
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 2);
-      for (int p = 0; p < 4; ++p) mbar_init(&sm.turn[i][p], 1);
       for (int bf = 0; bf < 2; ++bf) {
         mbar_init(&sm.s_full[i][bf], 1);
         mbar_init(&sm.p_ready[i][bf], kTile);
@@ -253,12 +251,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float sc2 = a.scale * kLog2e;
     bool ok = true;
     int hs = 0;    // half-steps of this tile done in earlier blocks (even)
-    // The two warps that share a scheduler (warp p of tile 0 and warp p of tile 1) take turns at the
-    // exponential loop, so that one tile's special-function work overlaps the other's TMEM loads,
-    // row maxima and barrier waits instead of both phases running in lockstep. Tile 0 goes first.
-    const int pair = warp & 3;
-    int turns = 0;  // turns taken so far (the same number on both tiles)
-    // Epilogues use the staging tile in a fixed order: per block tile 0, then tile 1.
     int nb = 0;                  // blocks this tile has finished
     int ep_base = 0;             // epilogues of earlier blocks
     bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
@@ -269,7 +261,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ep_base += 1;
         continue;
       }
-      const int shared_steps = bk.nkt1 ? 2 * bk.nkt0 : 0;   // half-steps that both tiles have
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;
       for (int t = 0; t < T && ok; ++t) {
@@ -324,11 +315,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         if (need) m_used = mx;
         const float neg_m = -m_used;
-        const bool take_turn = t < shared_steps;
-        if (take_turn && (w == 1 || turns > 0)) {
-          ok = mbar_wait(&sm.turn[w][pair], (w ? turns : turns - 1) & 1, abort_flag, a.status, code);
-          if (!ok) break;
-        }
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
@@ -342,11 +328,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             p[c2] = pack_bf16(p0, p1);
           }
           tmem_st16(s_addr + ch * 16, p);
-        }
-        if (take_turn) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.turn[w ^ 1][pair]);
-          ++turns;
         }
         tmem_wait_st();
         tc_fence_before();
@@ -391,7 +372,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       fence_proxy_async();
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(kTile) : "memory");
+      if (w == 0) asm volatile("bar.sync 1, 128;" ::: "memory");   // the 128 threads of this tile
+      else asm volatile("bar.sync 2, 128;" ::: "memory");
       if (row == 0) {
         tma_store_4d(&map_o, sm.o_stage, 0, h, bk.r0 + w * kTile, b);
         tma_store_4d(&map_o, sm.o_stage + kHalfBytes, 64, h, bk.r0 + w * kTile, b);

@@ -289,6 +289,301 @@ cudaError_t run_decode(const DecodeArgs& a, cudaStream_t s) {
   return e;
 }
 
+// ------------------------------------------------------------------ grouped-query heads on the tensor cores
+// With R >= 4 query heads per KV head the CUDA-core kernel above is bound by its multiply-adds
+// (every cache row is used R times), not by HBM. Here the R queries of a KV head are the rows
+// (padded to 16) of warp-level tensor-core MMAs: S = Q K^T over 32 cache rows at a time, online
+// softmax on the accumulator fragments, P (bf16) reused as the A operand of O += P V. Each of the
+// four consumer warps takes every fourth stage of the ring and keeps its own (m, l, O); the
+// states are merged at the end exactly as in the kernel above. Stages are [32 rows x 128] bf16
+// tiles of K and of V, loaded by TMA with the 128-byte swizzle so that ldmatrix is conflict-free.
+constexpr int kMmaWarps = 4;
+constexpr int kMmaThreads = (kMmaWarps + 1) * 32;
+constexpr int kMmaStages = 6;
+constexpr int kMmaRows = 32;                       // cache rows per stage
+constexpr int kMmaHalf = kMmaRows * 128;           // [32 rows x 64 bf16]
+
+struct MmaSmem {
+  alignas(1024) uint8_t k[kMmaStages][2 * kMmaHalf];
+  alignas(1024) uint8_t v[kMmaStages][2 * kMmaHalf];
+  uint64_t full[kMmaStages], empty[kMmaStages];
+  int abort_flag;
+};
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D += A B, A = 16 x 16 with rows 8..15 zero (a_lo: k 0..7, a_hi: k 8..15 of the thread's row), B = 16 x 8
+__device__ __forceinline__ void mma_16816(float* c, uint32_t a_lo, uint32_t a_hi, uint32_t b0, uint32_t b1) {
+  const uint32_t zero = 0;
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a_lo), "r"(zero), "r"(a_hi), "r"(zero), "r"(b0), "r"(b1));
+}
+
+// grid (splits, Hq / R, B), as decode_kernel. bf16, D = 128.
+template <int R>
+__global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                                  const __grid_constant__ CUtensorMap map_v,
+                                                                  DecodeArgs a) {
+  constexpr int D = 128;
+  constexpr int row_bytes = D * 2;
+  constexpr int NS = kMmaWarps + 1;                 // states to merge: one per warp + the appended row
+  extern __shared__ uint8_t smem_raw[];
+  MmaSmem& sm = *reinterpret_cast<MmaSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  float* red = reinterpret_cast<float*>(sm.k);      // [NS][R][D + 2], used once the ring has drained
+
+  const int split = blockIdx.x, hy = blockIdx.y, b = blockIdx.z;
+  const int h0 = hy * R;
+  const int rep = a.Hq / a.Hkv;
+  const int g = h0 / rep;
+  const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+  const int total = a.len + 1;
+  const int start = split * a.rows_per_split;
+  const int end = min(start + a.rows_per_split, total);
+  const int end_cached = min(end, a.len);
+  const int ncached = max(end_cached - start, 0);
+  const int nchunks = (ncached + kMmaRows - 1) / kMmaRows;
+  volatile int* abort_flag = &sm.abort_flag;
+
+  if (t == 0) {
+    for (int i = 0; i < kMmaStages; ++i) {
+      mbar_init(&sm.full[i], 1);
+      mbar_init(&sm.empty[i], 1);
+    }
+    sm.abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == kMmaWarps) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      prefetch_tensormap(&map_k);
+      prefetch_tensormap(&map_v);
+      bool ok = true;
+      for (int c = 0; c < nchunks && ok; ++c) {
+        const int st = c % kMmaStages;
+        if (c >= kMmaStages) ok = mbar_wait(&sm.empty[st], ((c / kMmaStages) - 1) & 1, abort_flag, a.status, PYR_ERR_TIMEOUT);
+        if (!ok) break;
+        const int row = start + c * kMmaRows;       // rows past the cache's capacity are zero fill
+        mbar_expect_tx(&sm.full[st], 4 * kMmaHalf);
+        tma_load_4d(sm.k[st], &map_k, &sm.full[st], 0, g, row, b);
+        tma_load_4d(sm.k[st] + kMmaHalf, &map_k, &sm.full[st], 64, g, row, b);
+        tma_load_4d(sm.v[st], &map_v, &sm.full[st], 0, g, row, b);
+        tma_load_4d(sm.v[st] + kMmaHalf, &map_v, &sm.full[st], 64, g, row, b);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ consumers
+    const int gq = lane >> 2, tq = lane & 3;        // fragment row (query) and column pair
+    const float sc2 = a.scale * kLog2e;
+    // A fragments of Q: row gq of the group (zero beyond R), d = 16 ks + 2 tq (+ 8)
+    uint32_t qa[8][2];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = qa[ks][1] = 0;
+      if (gq < R) {
+        const char* qrow = static_cast<const char*>(a.q) + ((size_t)b * a.Hq + h0 + gq) * row_bytes;
+        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + (ks * 16 + tq * 2) * 2);
+        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + (ks * 16 + 8 + tq * 2) * 2);
+      }
+    }
+    float m = -INFINITY, l = 0.f;                   // of row gq; l is this thread's share of the row sum
+    float o[16][4];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+    // ldmatrix: lane supplies row (lane & 7) of matrix (lane >> 3)
+    const int mi = lane >> 3, mr = lane & 7;
+
+    bool ok = true;
+    for (int c = warp; c < nchunks && ok; c += kMmaWarps) {
+      const int st = c % kMmaStages;
+      ok = mbar_wait(&sm.full[st], (c / kMmaStages) & 1, abort_flag, a.status, PYR_ERR_TIMEOUT);
+      if (!ok) break;
+      const int rows_here = min(kMmaRows, ncached - c * kMmaRows);
+      const uint32_t kb = smem_u32(sm.k[st]), vb = smem_u32(sm.v[st]);
+      if (rows_here < kMmaRows) {
+        // rows past the end of this split hold other data (or nothing): their scores are masked
+        // below, and their V must not reach the MMA as NaN or Inf
+        for (int i = lane; i < (kMmaRows - rows_here) * 16; i += 32) {
+          const int row = rows_here + (i >> 4), ch = i & 15;
+          *reinterpret_cast<uint4*>(sm.v[st] + (ch >> 3) * kMmaHalf + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
+              make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();
+      }
+      // S = Q K^T: 4 key tiles of 8
+      float sc[4][4];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+#pragma unroll
+      for (int kp = 0; kp < 2; ++kp) {
+        const int key = kp * 16 + (mi >> 1) * 8 + mr;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const int chunk = ks * 2 + (mi & 1);
+          uint32_t bf[4];
+          ldsm_x4(kb + (chunk >> 3) * kMmaHalf + key * 128 + (((chunk & 7) ^ (key & 7)) << 4), bf);
+          mma_16816(sc[2 * kp], qa[ks][0], qa[ks][1], bf[0], bf[1]);
+          mma_16816(sc[2 * kp + 1], qa[ks][0], qa[ks][1], bf[2], bf[3]);
+        }
+      }
+      // online softmax of row gq over the 32 keys (this thread: keys 8 nt + 2 tq, + 1)
+      float mx = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int key = nt * 8 + tq * 2 + e;
+          sc[nt][e] = key < rows_here ? sc[nt][e] * sc2 : -INFINITY;
+          mx = fmaxf(mx, sc[nt][e]);
+        }
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m, mx);             // finite: key 0 of a stage is always valid
+      const float corr = ex2(m - m_new);
+      float ps = 0.f;
+      uint32_t pa[2][2];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const float p0 = ex2(sc[nt][0] - m_new), p1 = ex2(sc[nt][1] - m_new);
+        ps += p0 + p1;
+        pa[nt >> 1][nt & 1] = pack_bf16(p0, p1);
+      }
+      l = l * corr + ps;
+      m = m_new;
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+      // O += P V: 2 steps of 16 keys, 16 tiles of 8 output columns
+#pragma unroll
+      for (int kp = 0; kp < 2; ++kp) {
+        const int key = kp * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+        for (int np = 0; np < 8; ++np) {
+          const int chunk = np * 2 + (mi >> 1);
+          uint32_t bf[4];
+          ldsm_x4_trans(vb + (chunk >> 3) * kMmaHalf + key * 128 + (((chunk & 7) ^ (key & 7)) << 4), bf);
+          mma_16816(o[2 * np], pa[kp][0], pa[kp][1], bf[0], bf[1]);
+          mma_16816(o[2 * np + 1], pa[kp][0], pa[kp][1], bf[2], bf[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.empty[st]);    // this warp is done reading the stage
+    }
+
+    // merge the warps' states and the appended row in a fixed order (the ring is idle by now)
+    asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory");
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (gq < R) {
+      float* dst = red + ((size_t)warp * R + gq) * (D + 2);
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) {
+        dst[nt * 8 + tq * 2] = o[nt][0];
+        dst[nt * 8 + tq * 2 + 1] = o[nt][1];
+      }
+      if (tq == 0) { dst[D] = m; dst[D + 1] = l; }
+    }
+    if (warp == 0) {
+      // the appended row, straight from k_new / v_new: a state with one key; the first head group
+      // of the KV head also stores it into the cache
+      const bool has_new = ok && end > a.len;
+      const char* kn = static_cast<const char*>(a.k_new) + ((size_t)b * a.Hkv + g) * row_bytes;
+      const char* vn = static_cast<const char*>(a.v_new) + ((size_t)b * a.Hkv + g) * row_bytes;
+      float kf[4] = {0.f, 0.f, 0.f, 0.f}, vf[4] = {0.f, 0.f, 0.f, 0.f};
+      if (has_new) {
+        const uint2 kr = *reinterpret_cast<const uint2*>(kn + lane * 8);
+        const uint2 vr = *reinterpret_cast<const uint2*>(vn + lane * 8);
+        if (h0 == g * rep) {
+          char* kc = static_cast<char*>(a.kc) + (((size_t)b * a.Hkv + g) * a.cap + a.len) * row_bytes;
+          char* vc = static_cast<char*>(a.vc) + (((size_t)b * a.Hkv + g) * a.cap + a.len) * row_bytes;
+          *reinterpret_cast<uint2*>(kc + lane * 8) = kr;
+          *reinterpret_cast<uint2*>(vc + lane * 8) = vr;
+        }
+        kf[0] = __uint_as_float(kr.x << 16); kf[1] = __uint_as_float(kr.x & 0xffff0000u);
+        kf[2] = __uint_as_float(kr.y << 16); kf[3] = __uint_as_float(kr.y & 0xffff0000u);
+        vf[0] = __uint_as_float(vr.x << 16); vf[1] = __uint_as_float(vr.x & 0xffff0000u);
+        vf[2] = __uint_as_float(vr.y << 16); vf[3] = __uint_as_float(vr.y & 0xffff0000u);
+      }
+      for (int r = 0; r < R; ++r) {
+        float* dst = red + ((size_t)kMmaWarps * R + r) * (D + 2);
+        float d = 0.f;
+        if (has_new) {
+          const uint2 qr = *reinterpret_cast<const uint2*>(static_cast<const char*>(a.q) +
+                                                           ((size_t)b * a.Hq + h0 + r) * row_bytes + lane * 8);
+          d = __uint_as_float(qr.x << 16) * kf[0] + __uint_as_float(qr.x & 0xffff0000u) * kf[1] +
+              __uint_as_float(qr.y << 16) * kf[2] + __uint_as_float(qr.y & 0xffff0000u) * kf[3];
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dst[lane * 4 + e] = vf[e];
+        if (lane == 0) { dst[D] = has_new ? d * sc2 : -INFINITY; dst[D + 1] = has_new ? 1.f : 0.f; }
+      }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory");
+    if (!*abort_flag) {
+      for (int i = t; i < R * D; i += kMmaWarps * 32) {
+        const int r = i / D, d = i % D;
+        float M = -INFINITY;
+        for (int gI = 0; gI < NS; ++gI) M = fmaxf(M, red[((size_t)gI * R + r) * (D + 2) + D]);
+        float num = 0.f, den = 0.f;
+        for (int gI = 0; gI < NS; ++gI) {
+          const float* src = red + ((size_t)gI * R + r) * (D + 2);
+          const float w = exp2f(src[D] - M);
+          num = fmaf(w, src[d], num);
+          den = fmaf(w, src[D + 1], den);
+        }
+        const int h = h0 + r;
+        if (a.splits == 1) {
+          static_cast<__nv_bfloat16*>(a.out)[((size_t)b * a.Hq + h) * D + d] = __float2bfloat16_rn(num / den);
+        } else {
+          const size_t pi = ((size_t)b * a.Hq + h) * a.splits + split;
+          a.part_acc[pi * D + d] = num;
+          if (d == 0) { a.part_ml[pi * 2] = M; a.part_ml[pi * 2 + 1] = den; }
+        }
+      }
+    }
+  }
+}
+
+template <int R>
+cudaError_t run_decode_mma(const DecodeArgs& a, cudaStream_t s) {
+  static_assert(sizeof(float) * (kMmaWarps + 1) * R * (128 + 2) <= sizeof(MmaSmem::k), "merge buffer fits in the K ring");
+  CUtensorMap mk, mv;
+  const int64_t sn = a.D, sh = (int64_t)a.cap * a.D, sb = (int64_t)a.Hkv * a.cap * a.D;
+  if (!make_tensor_map_bf16(&mk, a.kc, a.B, a.cap, a.Hkv, a.D, sb, sn, sh, kMmaRows) ||
+      !make_tensor_map_bf16(&mv, a.vc, a.B, a.cap, a.Hkv, a.D, sb, sn, sh, kMmaRows))
+    return cudaErrorInvalidValue;
+  constexpr size_t smem = sizeof(MmaSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(a.splits, a.Hq / R, a.B);
+  decode_mma_kernel<R><<<grid, kMmaThreads, smem, s>>>(mk, mv, a);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (a.splits > 1) {
+    decode_combine_kernel<__nv_bfloat16, 128><<<a.B * a.Hq, 128, 0, s>>>(a);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+// the tensor-core kernel needs TMA (16-byte aligned caches) and at least 4 query heads per KV head
+bool decode_mma_usable(const DecodeArgs& a) {
+  const int rep = a.Hq / a.Hkv;
+  return a.dtype == PYR_BF16 && a.D == 128 && rep % 4 == 0 && tensor_maps_available() &&
+         (reinterpret_cast<uintptr_t>(a.kc) | reinterpret_cast<uintptr_t>(a.vc)) % 16 == 0;
+}
+
 template <class T, int D>
 cudaError_t pick_r(const DecodeArgs& a, cudaStream_t s) {
   const int rep = a.Hq / a.Hkv;
@@ -301,6 +596,7 @@ cudaError_t pick_r(const DecodeArgs& a, cudaStream_t s) {
 }  // namespace
 
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s) {
+  if (decode_mma_usable(a)) return (a.Hq / a.Hkv) % 8 == 0 ? run_decode_mma<8>(a, s) : run_decode_mma<4>(a, s);
   if (a.dtype == PYR_F32) return a.D == 64 ? pick_r<float, 64>(a, s) : pick_r<float, 128>(a, s);
   return a.D == 64 ? pick_r<__nv_bfloat16, 64>(a, s) : pick_r<__nv_bfloat16, 128>(a, s);
 }

@@ -374,10 +374,10 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         if (!ok) break;
         const int row = start + c * kMmaRows;       // rows past the cache's capacity are zero fill
         mbar_expect_tx(&sm.full[st], 4 * kMmaHalf);
-        tma_load_4d(sm.k[st], &map_k, &sm.full[st], 0, g, row, b);
-        tma_load_4d(sm.k[st] + kMmaHalf, &map_k, &sm.full[st], 64, g, row, b);
-        tma_load_4d(sm.v[st], &map_v, &sm.full[st], 0, g, row, b);
-        tma_load_4d(sm.v[st] + kMmaHalf, &map_v, &sm.full[st], 64, g, row, b);
+        tma_load_4d(sm.k[st], &map_k, &sm.full[st], 0, row, g, b);
+        tma_load_4d(sm.k[st] + kMmaHalf, &map_k, &sm.full[st], 64, row, g, b);
+        tma_load_4d(sm.v[st], &map_v, &sm.full[st], 0, row, g, b);
+        tma_load_4d(sm.v[st] + kMmaHalf, &map_v, &sm.full[st], 64, row, g, b);
       }
     }
   } else {
@@ -559,9 +559,8 @@ template <int R>
 cudaError_t run_decode_mma(const DecodeArgs& a, cudaStream_t s) {
   static_assert(sizeof(float) * (kMmaWarps + 1) * R * (128 + 2) <= sizeof(MmaSmem::k), "merge buffer fits in the K ring");
   CUtensorMap mk, mv;
-  const int64_t sn = a.D, sh = (int64_t)a.cap * a.D, sb = (int64_t)a.Hkv * a.cap * a.D;
-  if (!make_tensor_map_bf16(&mk, a.kc, a.B, a.cap, a.Hkv, a.D, sb, sn, sh, kMmaRows) ||
-      !make_tensor_map_bf16(&mv, a.vc, a.B, a.cap, a.Hkv, a.D, sb, sn, sh, kMmaRows))
+  if (!make_tensor_map_rows_bf16(&mk, a.kc, a.B, a.Hkv, a.cap, a.D, kMmaRows) ||
+      !make_tensor_map_rows_bf16(&mv, a.vc, a.B, a.Hkv, a.cap, a.D, kMmaRows))
     return cudaErrorInvalidValue;
   constexpr size_t smem = sizeof(MmaSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -52,6 +52,20 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int B, int n, int 
   return r == CUDA_SUCCESS;
 }
 
+// Dense [batch][heads][rows][D] bf16 (the layer caches): coordinates are (x, row, head, batch).
+bool make_tensor_map_rows_bf16(CUtensorMap* map, const void* base, int batch, int heads, int rows, int D, int box_rows) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batch};
+  cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2, (cuuint64_t)heads * rows * D * 2};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 namespace {
 
 using namespace tc;

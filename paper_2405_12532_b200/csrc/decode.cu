@@ -294,12 +294,17 @@ cudaError_t run_decode(const DecodeArgs& a, cudaStream_t s) {
 // (every cache row is used R times), not by HBM. Here the R queries of a KV head are the rows
 // (padded to 16) of warp-level tensor-core MMAs: S = Q K^T over 32 cache rows at a time, online
 // softmax on the accumulator fragments, P (bf16) reused as the A operand of O += P V. Each of the
-// four consumer warps takes every fourth stage of the ring and keeps its own (m, l, O); the
-// states are merged at the end exactly as in the kernel above. Stages are [32 rows x 128] bf16
+// three consumer warps takes every third chunk and keeps its own (m, l, O); the states are merged
+// at the end exactly as in the kernel above. With six stages, stage c % 6 is only ever read by
+// warp c % 3, so every full/empty barrier has one waiter that follows it phase by phase. (A first
+// version with four warps let a warp meet a barrier it had skipped a phase of; a parity wait is
+// then ambiguous, a stage could be released early, and the producer's second expect_tx on a
+// barrier whose phase was still open faulted the kernel once loads completed out of order.) Stages are [32 rows x 128] bf16
 // tiles of K and of V, loaded by TMA with the 128-byte swizzle so that ldmatrix is conflict-free.
-constexpr int kMmaWarps = 4;
+constexpr int kMmaWarps = 3;
+static_assert(kMmaWarps * 2 == 6, "two stages per consumer warp");
 constexpr int kMmaThreads = (kMmaWarps + 1) * 32;
-constexpr int kMmaStages = 6;
+constexpr int kMmaStages = 2 * kMmaWarps;
 constexpr int kMmaRows = 32;                       // cache rows per stage
 constexpr int kMmaHalf = kMmaRows * 128;           // [32 rows x 64 bf16]
 

@@ -300,7 +300,8 @@ cudaError_t run_decode(const DecodeArgs& a, cudaStream_t s) {
 // version with four warps let a warp meet a barrier it had skipped a phase of; a parity wait is
 // then ambiguous, a stage could be released early, and the producer's second expect_tx on a
 // barrier whose phase was still open faulted the kernel once loads completed out of order.) Stages are [32 rows x 128] bf16
-// tiles of K and of V, loaded by TMA with the 128-byte swizzle so that ldmatrix is conflict-free.
+// tiles of K and of V, each one contiguous 8 KB TMA load (the rows are seen as half-rows of 128 bytes
+// with the 128-byte swizzle, which leaves ldmatrix with two-way bank conflicts instead of eight-way).
 constexpr int kMmaWarps = 3;
 static_assert(kMmaWarps * 2 == 6, "two stages per consumer warp");
 constexpr int kMmaThreads = (kMmaWarps + 1) * 32;
@@ -379,10 +380,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         if (!ok) break;
         const int row = start + c * kMmaRows;       // rows past the cache's capacity are zero fill
         mbar_expect_tx(&sm.full[st], 4 * kMmaHalf);
-        tma_load_4d(sm.k[st], &map_k, &sm.full[st], 0, row, g, b);
-        tma_load_4d(sm.k[st] + kMmaHalf, &map_k, &sm.full[st], 64, row, g, b);
-        tma_load_4d(sm.v[st], &map_v, &sm.full[st], 0, row, g, b);
-        tma_load_4d(sm.v[st] + kMmaHalf, &map_v, &sm.full[st], 64, row, g, b);
+        tma_load_4d(sm.k[st], &map_k, &sm.full[st], 0, 2 * row, g, b);   // 32 whole rows: 8 KB contiguous
+        tma_load_4d(sm.v[st], &map_v, &sm.full[st], 0, 2 * row, g, b);
       }
     }
   } else {
@@ -419,8 +418,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         // below, and their V must not reach the MMA as NaN or Inf
         for (int i = lane; i < (kMmaRows - rows_here) * 16; i += 32) {
           const int row = rows_here + (i >> 4), ch = i & 15;
-          *reinterpret_cast<uint4*>(sm.v[st] + (ch >> 3) * kMmaHalf + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
-              make_uint4(0, 0, 0, 0);
+          const int j = 2 * row + (ch >> 3);       // half-row
+          *reinterpret_cast<uint4*>(sm.v[st] + j * 128 + (((ch & 7) ^ (j & 7)) << 4)) = make_uint4(0, 0, 0, 0);
         }
         __syncwarp();
       }
@@ -435,7 +434,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         for (int ks = 0; ks < 8; ++ks) {
           const int chunk = ks * 2 + (mi & 1);
           uint32_t bf[4];
-          ldsm_x4(kb + (chunk >> 3) * kMmaHalf + key * 128 + (((chunk & 7) ^ (key & 7)) << 4), bf);
+          const int j = 2 * key + (chunk >> 3);    // half-row of the stage
+          ldsm_x4(kb + j * 128 + (((chunk & 7) ^ (j & 7)) << 4), bf);
           mma_16816(sc[2 * kp], qa[ks][0], qa[ks][1], bf[0], bf[1]);
           mma_16816(sc[2 * kp + 1], qa[ks][0], qa[ks][1], bf[2], bf[3]);
         }
@@ -475,7 +475,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         for (int np = 0; np < 8; ++np) {
           const int chunk = np * 2 + (mi >> 1);
           uint32_t bf[4];
-          ldsm_x4_trans(vb + (chunk >> 3) * kMmaHalf + key * 128 + (((chunk & 7) ^ (key & 7)) << 4), bf);
+          const int j = 2 * key + (chunk >> 3);
+          ldsm_x4_trans(vb + j * 128 + (((chunk & 7) ^ (j & 7)) << 4), bf);
           mma_16816(o[2 * np], pa[kp][0], pa[kp][1], bf[0], bf[1]);
           mma_16816(o[2 * np + 1], pa[kp][0], pa[kp][1], bf[2], bf[3]);
         }
@@ -564,8 +565,8 @@ template <int R>
 cudaError_t run_decode_mma(const DecodeArgs& a, cudaStream_t s) {
   static_assert(sizeof(float) * (kMmaWarps + 1) * R * (128 + 2) <= sizeof(MmaSmem::k), "merge buffer fits in the K ring");
   CUtensorMap mk, mv;
-  if (!make_tensor_map_rows_bf16(&mk, a.kc, a.B, a.Hkv, a.cap, a.D, kMmaRows) ||
-      !make_tensor_map_rows_bf16(&mv, a.vc, a.B, a.Hkv, a.cap, a.D, kMmaRows))
+  if (!make_tensor_map_rows_bf16(&mk, a.kc, a.B, a.Hkv, a.cap, kMmaRows) ||
+      !make_tensor_map_rows_bf16(&mv, a.vc, a.B, a.Hkv, a.cap, kMmaRows))
     return cudaErrorInvalidValue;
   constexpr size_t smem = sizeof(MmaSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

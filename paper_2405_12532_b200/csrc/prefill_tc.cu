@@ -52,13 +52,15 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int B, int n, int 
   return r == CUDA_SUCCESS;
 }
 
-// Dense [batch][heads][rows][D] bf16 (the layer caches): coordinates are (x, row, head, batch).
-bool make_tensor_map_rows_bf16(CUtensorMap* map, const void* base, int batch, int heads, int rows, int D, int box_rows) {
+// Dense [batch][heads][rows][128] bf16 (the layer caches), seen as 2 * rows half-rows of 64 elements so
+// that one box of 2 * box_rows half-rows is box_rows whole rows, contiguous in memory:
+// coordinates are (0, 2 * row, head, batch); half-row j lands at offset 128 j, 16-byte chunk c at c ^ (j & 7).
+bool make_tensor_map_rows_bf16(CUtensorMap* map, const void* base, int batch, int heads, int rows, int box_rows) {
   EncodeFn enc = encode_fn();
   if (!enc) return false;
-  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batch};
-  cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2, (cuuint64_t)heads * rows * D * 2};
-  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  cuuint64_t dims[4] = {64, (cuuint64_t)rows * 2, (cuuint64_t)heads, (cuuint64_t)batch};
+  cuuint64_t strides[3] = {128, (cuuint64_t)rows * 256, (cuuint64_t)heads * rows * 256};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows * 2, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

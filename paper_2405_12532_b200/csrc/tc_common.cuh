@@ -244,7 +244,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 bool tensor_maps_available();   // the driver's tensor-map encoder could be resolved
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int B, int n, int H, int D, int64_t sb, int64_t sn,
                           int64_t sh, int box_rows);
-// Dense [batch][heads][rows][D] bf16: 64-column boxes of `box_rows` rows, coordinates (x, row, head, batch).
-bool make_tensor_map_rows_bf16(CUtensorMap* map, const void* base, int batch, int heads, int rows, int D, int box_rows);
+// Dense [batch][heads][rows][128] bf16 seen as half-rows of 64 elements: a box is `box_rows` whole rows,
+// contiguous in memory; coordinates (0, 2 * row, head, batch); half-row j at offset 128 j, swizzled by j & 7.
+bool make_tensor_map_rows_bf16(CUtensorMap* map, const void* base, int batch, int heads, int rows, int box_rows);
 
 }  // namespace pyr

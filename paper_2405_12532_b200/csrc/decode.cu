@@ -405,6 +405,18 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
     for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     // ldmatrix: lane supplies row (lane & 7) of matrix (lane >> 3)
     const int mi = lane >> 3, mr = lane & 7;
+    // Byte offsets of this lane's ldmatrix rows inside a stage, without the 16-key step (4096 bytes).
+    // A stage holds half-rows of 128 bytes: half-row j = 2 * key + (d >= 64), 16-byte chunk c at c ^ (j & 7).
+    uint32_t koff[8], voff[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // K (plain): matrices (keys 0-7, d lo) (keys 0-7, d hi) (keys 8-15, d lo) (keys 8-15, d hi) of k-step i
+      koff[i] = (uint32_t)((2 * ((mi >> 1) * 8 + mr) + (i >> 2)) * 128 +
+                           ((((i & 3) * 2 + (mi & 1)) ^ ((2 * mr + (i >> 2)) & 7)) << 4));
+      // V (transposed): matrices (keys 0-7, d lo) (keys 8-15, d lo) (keys 0-7, d hi) (keys 8-15, d hi) of column pair i
+      voff[i] = (uint32_t)((2 * ((mi & 1) * 8 + mr) + (i >> 2)) * 128 +
+                           ((((i & 3) * 2 + (mi >> 1)) ^ ((2 * mr + (i >> 2)) & 7)) << 4));
+    }
 
     bool ok = true;
     for (int c = warp; c < nchunks && ok; c += kMmaWarps) {
@@ -429,13 +441,10 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
       for (int nt = 0; nt < 4; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
 #pragma unroll
       for (int kp = 0; kp < 2; ++kp) {
-        const int key = kp * 16 + (mi >> 1) * 8 + mr;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          const int chunk = ks * 2 + (mi & 1);
           uint32_t bf[4];
-          const int j = 2 * key + (chunk >> 3);    // half-row of the stage
-          ldsm_x4(kb + j * 128 + (((chunk & 7) ^ (j & 7)) << 4), bf);
+          ldsm_x4(kb + kp * 4096 + koff[ks], bf);
           mma_16816(sc[2 * kp], qa[ks][0], qa[ks][1], bf[0], bf[1]);
           mma_16816(sc[2 * kp + 1], qa[ks][0], qa[ks][1], bf[2], bf[3]);
         }
@@ -446,8 +455,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
       for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int key = nt * 8 + tq * 2 + e;
-          sc[nt][e] = key < rows_here ? sc[nt][e] * sc2 : -INFINITY;
+          sc[nt][e] *= sc2;
+          if (rows_here < kMmaRows && nt * 8 + tq * 2 + e >= rows_here) sc[nt][e] = -INFINITY;
           mx = fmaxf(mx, sc[nt][e]);
         }
       }
@@ -465,18 +474,17 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
       }
       l = l * corr + ps;
       m = m_new;
+      if (__any_sync(0xffffffffu, corr != 1.f)) {    // once the maxima have settled there is nothing to rescale
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+      }
       // O += P V: 2 steps of 16 keys, 16 tiles of 8 output columns
 #pragma unroll
       for (int kp = 0; kp < 2; ++kp) {
-        const int key = kp * 16 + (mi & 1) * 8 + mr;
 #pragma unroll
         for (int np = 0; np < 8; ++np) {
-          const int chunk = np * 2 + (mi >> 1);
           uint32_t bf[4];
-          const int j = 2 * key + (chunk >> 3);
-          ldsm_x4_trans(vb + j * 128 + (((chunk & 7) ^ (j & 7)) << 4), bf);
+          ldsm_x4_trans(vb + kp * 4096 + voff[np], bf);
           mma_16816(o[2 * np], pa[kp][0], pa[kp][1], bf[0], bf[1]);
           mma_16816(o[2 * np + 1], pa[kp][0], pa[kp][1], bf[2], bf[3]);
         }

@@ -57,17 +57,9 @@ extern "C" pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new
   a.B = batch; a.Hq = n_q_heads; a.Hkv = n_kv_heads; a.D = head_dim;
   a.len = len; a.cap = cap; a.dtype = dtype;
   a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
-  // same split rule as pyr_decode_attn: fill the machine a few times over
-  const int total = len + 1;
-  const long long pairs = (long long)batch * n_kv_heads;
-  int splits = (int)((148LL * 8 + pairs - 1) / pairs);
-  const int max_by_rows = (total + 127) / 128;
-  if (splits > max_by_rows) splits = max_by_rows;
-  if (splits > pyr::kMaxDecodeSplits) splits = pyr::kMaxDecodeSplits;
-  if (splits < 1) splits = 1;
-  int rps = (total + splits - 1) / splits;
-  rps = (rps + 15) / 16 * 16;
-  splits = (total + rps - 1) / rps;
+  // same split rule as pyr_decode_attn
+  int splits = 1, rps = 0;
+  pyr::decode_split_rule(batch, n_kv_heads, len + 1, &splits, &rps);
   a.splits = splits; a.rows_per_split = rps;
 
   a.part_acc = nullptr; a.part_ml = nullptr;

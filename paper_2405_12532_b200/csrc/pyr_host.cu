@@ -401,17 +401,8 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   a.len = c->len_now[layer]; a.cap = p.cap;
   a.scale = c->scale; a.dtype = c->cfg.dtype;
   a.status = at<int>(c, c->lay.status);
-  // Split the rows so that the grid fills the machine a few times over.
-  const int total = a.len + 1;
-  const long long pairs = (long long)a.B * a.Hkv;
-  int splits = (int)((148LL * 8 + pairs - 1) / pairs);
-  const int max_by_rows = (total + 127) / 128;
-  if (splits > max_by_rows) splits = max_by_rows;
-  if (splits > pyr::kMaxDecodeSplits) splits = pyr::kMaxDecodeSplits;
-  if (splits < 1) splits = 1;
-  int rps = (total + splits - 1) / splits;
-  rps = (rps + 15) / 16 * 16;
-  splits = (total + rps - 1) / rps;
+  int splits = 1, rps = 0;
+  pyr::decode_split_rule(a.B, a.Hkv, a.len + 1, &splits, &rps);
   a.splits = splits; a.rows_per_split = rps;
   if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
   g_launches += splits > 1 ? 2 : 1;

@@ -58,6 +58,22 @@ struct DecodeArgs {
   int* status;                     // device status word, may be null
 };
 
+// Split-K rule of the decode kernels: rows [0, total) of a cache are cut into `splits` ranges of
+// `rows_per_split` (a multiple of 16) so that the grid is about one full wave of two CTAs per SM;
+// the kernels are bandwidth-bound, and on short caches more, smaller CTAs only add fixed costs.
+inline void decode_split_rule(int batch, int n_kv_heads, int total, int* splits_out, int* rows_per_split_out) {
+  const long long pairs = (long long)batch * n_kv_heads;
+  int splits = (int)((148LL * 2 + pairs - 1) / pairs);
+  const int max_by_rows = (total + 127) / 128;
+  if (splits > max_by_rows) splits = max_by_rows;
+  if (splits > kMaxDecodeSplits) splits = kMaxDecodeSplits;
+  if (splits < 1) splits = 1;
+  int rps = (total + splits - 1) / splits;
+  rps = (rps + 15) / 16 * 16;
+  *splits_out = (total + rps - 1) / rps;
+  *rows_per_split_out = rps;
+}
+
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s);     // bf16, D = 128, tcgen05

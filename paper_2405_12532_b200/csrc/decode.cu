@@ -314,7 +314,6 @@ struct MmaSmem {
   alignas(1024) uint8_t v[kMmaStages][2 * kMmaHalf];
   uint64_t full[kMmaStages], empty[kMmaStages];
   int abort_flag;
-  int is_last;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t* r) {
@@ -567,39 +566,6 @@ __global__ void __launch_bounds__(kMmaThreads) decode_mma_kernel(const __grid_co
         }
       }
     }
-    if (a.splits > 1 && a.counters) {
-      // The CTA that finishes last among the splits of this head group merges them (ascending
-      // split order, the arithmetic of decode_combine_kernel) and leaves the counter at zero.
-      __threadfence();
-      asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory");
-      if (t == 0) {
-        __threadfence();
-        const int seen = atomicAdd(&a.counters[b * gridDim.y + hy], 1);
-        __threadfence();
-        sm.is_last = (seen == a.splits - 1);
-      }
-      asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory");
-      if (sm.is_last) {
-        if (!a.status || !*reinterpret_cast<volatile int*>(a.status)) {
-          for (int i = t; i < R * D; i += kMmaWarps * 32) {
-            const int r = i / D, d = i % D;
-            const size_t bh = (size_t)b * a.Hq + h0 + r;
-            const float* ml = a.part_ml + bh * a.splits * 2;
-            const float* pa = a.part_acc + bh * a.splits * D;
-            float M = -INFINITY;
-            for (int sp = 0; sp < a.splits; ++sp) M = fmaxf(M, __ldcg(ml + sp * 2));
-            float num = 0.f, den = 0.f;
-            for (int sp = 0; sp < a.splits; ++sp) {
-              const float w = exp2f(__ldcg(ml + sp * 2) - M);
-              num = fmaf(w, __ldcg(pa + (size_t)sp * D + d), num);
-              den = fmaf(w, __ldcg(ml + sp * 2 + 1), den);
-            }
-            static_cast<__nv_bfloat16*>(a.out)[bh * D + d] = __float2bfloat16_rn(num / den);
-          }
-        }
-        if (t == 0) a.counters[b * gridDim.y + hy] = 0;
-      }
-    }
   }
 }
 
@@ -617,7 +583,7 @@ cudaError_t run_decode_mma(const DecodeArgs& a, cudaStream_t s) {
   decode_mma_kernel<R><<<grid, kMmaThreads, smem, s>>>(mk, mv, a);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (a.splits > 1 && !a.counters) {
+  if (a.splits > 1) {
     decode_combine_kernel<__nv_bfloat16, 128><<<a.B * a.Hq, 128, 0, s>>>(a);
     e = cudaGetLastError();
   }
@@ -641,11 +607,6 @@ cudaError_t pick_r(const DecodeArgs& a, cudaStream_t s) {
 }
 
 }  // namespace
-
-int decode_launches(const DecodeArgs& a) {
-  if (a.splits <= 1) return 1;
-  return decode_mma_usable(a) && a.counters ? 1 : 2;
-}
 
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s) {
   if (decode_mma_usable(a)) return (a.Hq / a.Hkv) % 8 == 0 ? run_decode_mma<8>(a, s) : run_decode_mma<4>(a, s);

@@ -64,7 +64,6 @@ extern "C" pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new
 
   a.part_acc = nullptr; a.part_ml = nullptr;
   a.status = nullptr;
-  a.counters = nullptr;           // the splits are merged by the second kernel
   if (splits > 1) {
     const size_t acc_floats = (size_t)batch * n_q_heads * splits * head_dim;
     const size_t ml_floats = (size_t)batch * n_q_heads * splits * 2;

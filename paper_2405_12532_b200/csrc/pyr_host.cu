@@ -24,7 +24,7 @@ constexpr size_t kAlign = 256;
 std::atomic<uint64_t> g_launches{0};   // kernels launched by this process through the library
 
 struct Layout {
-  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, dec_counters, total;
+  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, total;
   std::vector<LayerPlan> layers;
 };
 
@@ -80,8 +80,6 @@ void plan(const pyr_config_t* c, Layout* lay) {
   if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * D * 4, kAlign);
   lay->part_ml = off;
   if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * 2 * 4, kAlign);
-  lay->dec_counters = off;       // arrival counters of the split-K merge, zero between launches
-  if (c->max_new_tokens > 0) off = align_up(off + B * Hq * 4, kAlign);
   lay->layers.resize(c->n_layers);
   int n_in = N;
   for (int l = 0; l < c->n_layers; ++l) {
@@ -131,9 +129,6 @@ T* at(const pyr_cache* c, size_t off) { return reinterpret_cast<T*>(c->base + of
 
 pyr_status_t device_init(pyr_cache* c, cudaStream_t s) {
   if (cudaMemsetAsync(at<int>(c, c->lay.status), 0, pyr::kStatusWords * sizeof(int), s) != cudaSuccess)
-    return PYR_ERR_CUDA;
-  if (c->cfg.max_new_tokens > 0 &&
-      cudaMemsetAsync(at<int>(c, c->lay.dec_counters), 0, (size_t)c->cfg.batch * c->cfg.n_q_heads * 4, s) != cudaSuccess)
     return PYR_ERR_CUDA;
   if (c->needs_init) {
     int dev = 0, major = 0;
@@ -406,12 +401,11 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   a.len = c->len_now[layer]; a.cap = p.cap;
   a.scale = c->scale; a.dtype = c->cfg.dtype;
   a.status = at<int>(c, c->lay.status);
-  a.counters = at<int>(c, c->lay.dec_counters);
   int splits = 1, rps = 0;
   pyr::decode_split_rule(a.B, a.Hkv, a.len + 1, &splits, &rps);
   a.splits = splits; a.rows_per_split = rps;
   if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
-  g_launches += pyr::decode_launches(a);
+  g_launches += splits > 1 ? 2 : 1;
   c->len_now[layer] += 1;
   return PYR_OK;
 }

@@ -56,7 +56,6 @@ struct DecodeArgs {
   float scale;
   int dtype;
   int* status;                     // device status word, may be null
-  int* counters;                   // [B, Hq] zeroed ints or null: lets the last CTA of a head group merge the splits
 };
 
 // Split-K rule of the decode kernels: rows [0, total) of a cache are cut into `splits` ranges of
@@ -88,6 +87,5 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s);
 cudaError_t launch_compact_rows(const RowsArgs& a, cudaStream_t s);
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s);
-int decode_launches(const DecodeArgs& a);   // kernels launch_decode starts for these arguments (1 or 2)
 
 }  // namespace pyr

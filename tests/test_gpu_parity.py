@@ -245,7 +245,9 @@ def test_hidden_rows_compaction_wide():
 # ---------------------------------------------------------------- decode over longer caches (split-K)
 @pytest.mark.parametrize("dtype,Hq,Hkv,D,B,n", [("bf16", 8, 1, 128, 2, 3000), ("bf16", 4, 4, 128, 3, 1111),
                                                  ("f32", 4, 2, 128, 1, 900), ("bf16", 6, 3, 64, 2, 517),
-                                                 ("f32", 3, 3, 64, 2, 140), ("bf16", 16, 2, 128, 1, 2500)])
+                                                 ("f32", 3, 3, 64, 2, 140), ("bf16", 16, 2, 128, 1, 2500),
+                                                 # 8 heads per KV head, splits long enough to wrap the stage ring
+                                                 ("bf16", 64, 8, 128, 4, 6000), ("bf16", 8, 2, 128, 24, 3333)])
 def test_decode_split_k(dtype, Hq, Hkv, D, B, n):
     L, T = 32, 3
     w = dict(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, sel_groups=Hkv, dtype=dtype, batch=B,

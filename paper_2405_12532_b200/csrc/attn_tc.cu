@@ -61,7 +61,7 @@ struct AttnSmem {
 struct Block {
   int r0, nkt0, nkt1, nkt;   // first row; key tiles of tile 0 / tile 1 (0 = tile absent) / loaded
 };
-__device__ __forceinline__ Block block_of(int blk, int n) {
+__host__ __device__ __forceinline__ Block block_of(int blk, int n) {
   const int ntiles = (n + kTile - 1) / kTile;
   Block b;
   if (ntiles & 1) {
@@ -77,18 +77,29 @@ __device__ __forceinline__ Block block_of(int blk, int n) {
   return b;
 }
 
+// A head's blocks can be dealt to `parts` CTAs (used when there are too few heads to fill the SMs
+// evenly). With the blocks numbered from the longest (k = 0), part p takes k = p, 2 parts - 1 - p,
+// 2 parts + p, 4 parts - 1 - p, ...: a long block is paired with a short one, so the parts carry
+// nearly equal work. Returns false when part `part` has no it-th block.
+__host__ __device__ __forceinline__ bool block_at(int it, int part, int parts, int n, Block* bk) {
+  const int nblk = (n + 2 * kTile - 1) / (2 * kTile);
+  const int k = 2 * parts * (it >> 1) + ((it & 1) ? 2 * parts - 1 - part : part);
+  if (k >= nblk) return false;
+  *bk = block_of(nblk - 1 - k, n);
+  return true;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
-               PrefillArgs a) {
+               PrefillArgs a, int parts) {
   extern __shared__ uint8_t smem_raw[];
   AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-  const int h = blockIdx.x, b = blockIdx.y;
+  const int h = blockIdx.x / parts, part = blockIdx.x % parts, b = blockIdx.y;
   const int g = h / (a.Hq / a.Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = a.n;
-  const int nblk = (n + 2 * kTile - 1) / (2 * kTile);
   volatile int* abort_flag = &sm.abort_flag;
   if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
@@ -129,8 +140,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bool ok = true;
       int kv = 0;                                      // K/V tiles loaded so far (stage = kv & 1)
       int nq[2] = {0, 0};                              // Q loads issued per tile
-      for (int it = 0; it < nblk && ok; ++it) {
-        const Block bk = block_of(nblk - 1 - it, n);   // longest block first
+      for (int it = 0; ok; ++it) {
+        Block bk;
+        if (!block_at(it, part, parts, n, &bk)) break;   // longest block first
         for (int w = 0; w < 2 && ok; ++w) {
           if (w == 1 && !bk.nkt1) break;
           // the S MMAs of the previous block have finished reading this Q tile
@@ -177,8 +189,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int kvu = 0;   // K/V tiles of the ring that earlier blocks used
       int nq = 0;    // Q loads of this tile consumed
       int hs = 0;    // half-steps of this tile done in earlier blocks (even)
-      for (int it = 0; it < nblk && ok; ++it) {
-        const Block bk = block_of(nblk - 1 - it, n);
+      for (int it = 0; ok; ++it) {
+        Block bk;
+        if (!block_at(it, part, parts, n, &bk)) break;
         const int nkt_w = w ? bk.nkt1 : bk.nkt0;
         const int T = 2 * nkt_w;
         // when the key tiles come in descending order, the one tile 0 does not read comes first
@@ -254,8 +267,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     int nb = 0;                  // blocks this tile has finished
     int ep_base = 0;             // epilogues of earlier blocks
     bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
-    for (int it = 0; it < nblk && ok; ++it) {
-      const Block bk = block_of(nblk - 1 - it, n);
+    for (int it = 0; ok; ++it) {
+      Block bk;
+      if (!block_at(it, part, parts, n, &bk)) break;
       const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
       if (T == 0) {
         ep_base += 1;
@@ -419,8 +433,29 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   const size_t smem = sizeof(AttnSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(a.Hq, a.B);
-  attn_tc_kernel<<<grid, kThreads, smem, s>>>(mq, mk, mv, mo, a);
+  // One CTA per (sequence, head) when that fills the SMs evenly; otherwise deal each head's blocks
+  // to 2, 4 or 8 CTAs. Cost model: waves of CTAs x the largest share of key-tile steps a CTA gets
+  // (a block costs about one step more, a CTA about two); splitting must win by 5 % to be chosen.
+  int dev = 0, sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const int nblk = (a.n + 2 * kTile - 1) / (2 * kTile);
+  const long long heads = (long long)a.Hq * a.B;
+  int parts = 1;
+  long long best = -1;
+  for (int p = 1; p <= 8 && p <= nblk; p *= 2) {
+    long long share = 0;                       // key-tile steps of the busiest part
+    for (int part = 0; part < p; ++part) {
+      long long w = 0;
+      Block bk;
+      for (int it = 0; block_at(it, part, p, a.n, &bk); ++it) w += bk.nkt + 1;
+      if (w + 2 > share) share = w + 2;
+    }
+    const long long cost = ((heads * p + sms - 1) / sms) * share;
+    if (best < 0 || cost * 100 < best * 95) { best = cost; parts = p; }
+  }
+  dim3 grid(a.Hq * parts, a.B);
+  attn_tc_kernel<<<grid, kThreads, smem, s>>>(mq, mk, mv, mo, a, parts);
   return cudaGetLastError();
 }
 

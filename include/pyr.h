@@ -111,8 +111,9 @@ pyr_status_t pyr_cache_layer_info(const pyr_cache_t* cache, int32_t layer, int32
 
 /* Size and alignment of the device buffer pyr_cache_alloc needs for `cfg`
  * (Section 4.1: each layer's cache holds only its PvC and window, plus T
- * decode rows; the buffer also holds scores, lse, kept indices, positions, the
- * decode workspace and the status word). Validates cfg. */
+ * decode rows; the buffer also holds scores (pooled, and per head for the
+ * tensor-core score pass), lse, kept indices, positions, the decode workspace
+ * and the status word). Validates cfg. */
 pyr_status_t pyr_cache_bytes(const pyr_config_t* cfg, size_t* bytes, size_t* align);
 
 /* Builds a cache handle over the caller's device buffer `dev_buf` (device,

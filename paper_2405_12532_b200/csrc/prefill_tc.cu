@@ -147,7 +147,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int i = 0; i < kScoreBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.s_empty[i], kScoreGroups * kTile);
+      mbar_init(&sm.s_empty[i], kScoreCompute);      // one arrival per compute warp
     }
     sm.abort_flag = 0;
     fence_barrier_init();
@@ -267,7 +267,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
         tmem_wait_ld();
         tc_fence_before();
-        mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);   // 512 arrivals on one word would serialise
       };
       auto weigh = [&](const uint32_t* r, int qt) -> float {
         const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 32]);

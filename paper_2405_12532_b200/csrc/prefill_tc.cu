@@ -87,15 +87,12 @@ enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 // from one item into the next: one lane of warp 9 issues the TMA loads. Per
 // (key tile, query tile) step one lane of warp 8 issues
 // S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one of four TMEM
-// buffers. Sixteen compute warps in four groups: group g takes query columns
-// 32 g .. 32 g + 31 of every step; a thread owns one key and sums
-// w_i * exp(s_ij - lse_i) over its columns of every query tile, then writes the
-// key's partial score of (head, query chunk, column group). Four warps per
-// scheduler keep the special-function unit busy while others wait or load. A
-// second kernel adds the partial scores of a selection group in a fixed order.
-constexpr int kScoreGroups = 4;                        // column groups of 32 queries
-constexpr int kScoreCompute = kScoreGroups * 4;        // compute warps; then the MMA warp, then the TMA warp
-constexpr int kScoreThreads = (kScoreCompute + 2) * 32;
+// buffers. Warps 0-3 take query columns 0..63 of the step, warps
+// 4-7 columns 64..127; a thread owns one key and sums w_i * exp(s_ij - lse_i)
+// over its columns of every query tile, then writes the key's partial score of
+// (head, query chunk, column half). A second kernel adds the partial scores of
+// a selection group in a fixed order.
+constexpr int kScoreThreads = 320;
 constexpr int kScoreBufs = 4;              // TMEM buffers of 128 columns
 constexpr int kMaxQTiles = 4;              // query tiles resident per item
 constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
@@ -147,12 +144,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int i = 0; i < kScoreBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.s_empty[i], kScoreCompute);      // one arrival per compute warp
+      mbar_init(&sm.s_empty[i], 2 * kTile);
     }
     sm.abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == kScoreCompute) {
+  if (warp == 8) {
     tmem_alloc(&sm.tmem_base, kScoreBufs * kTile);
     tmem_relinquish();
   }
@@ -161,7 +158,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp == kScoreCompute + 1) {
+  if (warp == 9) {
     // ---------------------------------------------------------------- TMA loads
     if (lane == 0 && my_items > 0) {
       prefetch_tensormap(&map_q);
@@ -192,7 +189,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == kScoreCompute) {
+  } else if (warp == 8) {
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0 && my_items > 0) {
       constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
@@ -228,53 +225,62 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     __syncwarp();
   } else {
-    const int wg = warp >> 2;                 // column group of every step
+    const int wg = warp >> 2;                 // column half of every step
     const int key = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float sc2 = a.scale * kLog2e;
     // bias of recent query i: log2 w_i - lse_i log2 e; -inf beyond the window (those Q rows are zero fill).
-    // A thread fetches its entry of the next item while it works on this one.
+    // A thread fetches its (at most two) entries of the next item while it works on this one.
     auto bias_of = [&](const ScoreItem& it, int i) -> float {
       const int qi = it.q0 + i;
       return (i < it.nq * kTile && qi < L)
                  ? log2f(a.w[qi]) - a.lse[((int64_t)it.b * a.Hq + it.h) * n + c + qi] * kLog2e
                  : -INFINITY;
     };
-    static_assert(kScoreGroups * kTile == kMaxQTiles * kTile, "one bias entry per compute thread");
-    float nb = my_items > 0 ? bias_of(item_of(0), threadIdx.x) : 0.f;
+    float nb0 = 0.f, nb1 = 0.f;
+    if (my_items > 0) {
+      const ScoreItem it = item_of(0);
+      nb0 = bias_of(it, threadIdx.x);
+      nb1 = bias_of(it, threadIdx.x + 2 * kTile);
+    }
     bool ok = true;
     int sg = 0;   // steps of earlier items
     for (int k = 0; k < my_items && ok; ++k) {
       const ScoreItem it = item_of(k);
       float* bias = sm.bias[k & 1];
-      bias[threadIdx.x] = nb;
+      bias[threadIdx.x] = nb0;
+      bias[threadIdx.x + 2 * kTile] = nb1;
       // every thread is past its reads of this buffer (item k - 2) since it went through the barrier of item k - 1
-      asm volatile("bar.sync 1, %0;" ::"n"(kScoreGroups * kTile) : "memory");
-      if (k + 1 < my_items) nb = bias_of(item_of(k + 1), threadIdx.x);
-      float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * kScoreGroups * (int64_t)c + (int64_t)wg * c;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (k + 1 < my_items) {
+        const ScoreItem nx = item_of(k + 1);
+        nb0 = bias_of(nx, threadIdx.x);
+        nb1 = bias_of(nx, threadIdx.x + 2 * kTile);
+      }
+      float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * 2 * (int64_t)c + (int64_t)wg * c;
       const int nq = it.nq;
       const int steps = nkt * nq;
       // The TMEM load of step s+1 is issued before the exponentials of step s, so that its latency
       // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
-      uint32_t ra[32], rb[32];
+      uint32_t ra[64], rb[64];
       auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
         const int buf = (sg + s) & (kScoreBufs - 1);
         ok = mbar_wait(&sm.s_full[buf], ((sg + s) / kScoreBufs) & 1, abort_flag, a.status, kTimeoutScore);
         if (!ok) return;
         tc_fence_after();
-        tmem_ld32(tmem + lane_base + buf * kTile + wg * 32, r);
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
+        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
       };
       auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
         tmem_wait_ld();
         tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);   // 512 arrivals on one word would serialise
+        mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);
       };
       auto weigh = [&](const uint32_t* r, int qt) -> float {
-        const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 32]);
+        const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 64]);
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
+        for (int c4 = 0; c4 < 16; ++c4) {
           const float4 bv = bias4[c4];
           part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
           part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
@@ -312,7 +318,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kScoreCompute) {
+  if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem, kScoreBufs * kTile);
   }
@@ -337,7 +343,6 @@ bool score_tc_supported(const PrefillArgs& a) {
 }
 bool tensor_maps_available() { return encode_fn() != nullptr; }
 
-int score_tc_groups() { return kScoreGroups; }
 int score_tc_chunks(int L) { return ((L + kTile - 1) / kTile + kMaxQTiles - 1) / kMaxQTiles; }
 
 cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s) {
@@ -361,7 +366,7 @@ cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s
   if (e != cudaSuccess) return e;
   const int heads = a.Hq / a.G;
   dim3 rgrid((c + 255) / 256, a.G, a.B);
-  score_reduce_kernel<<<rgrid, 256, 0, s>>>(partial, a.score, c, a.G, heads * nchunk * kScoreGroups, heads, a.status);
+  score_reduce_kernel<<<rgrid, 256, 0, s>>>(partial, a.score, c, a.G, heads * nchunk * 2, heads, a.status);
   return cudaGetLastError();
 }
 

@@ -87,11 +87,12 @@ enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 // from one item into the next: one lane of warp 9 issues the TMA loads. Per
 // (key tile, query tile) step one lane of warp 8 issues
 // S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one of four TMEM
-// buffers. Warps 0-3 take query columns 0..63 of the step, warps
-// 4-7 columns 64..127; a thread owns one key and sums w_i * exp(s_ij - lse_i)
-// over its columns of every query tile, then writes the key's partial score of
-// (head, query chunk, column half). A second kernel adds the partial scores of
-// a selection group in a fixed order.
+// buffers. Warps 0-3 take the even steps, warps 4-7 the odd ones (so the two
+// warps that share a scheduler are never in the same phase and the
+// special-function unit stays busy); a thread owns one key and sums
+// w_i * exp(s_ij - lse_i) over the 128 query columns of its steps, then writes
+// the key's partial score of (head, query chunk, step parity). A second kernel
+// adds the partial scores of a selection group in a fixed order.
 constexpr int kScoreThreads = 320;
 constexpr int kScoreBufs = 4;              // TMEM buffers of 128 columns
 constexpr int kMaxQTiles = 4;              // query tiles resident per item
@@ -144,7 +145,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int i = 0; i < kScoreBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.s_empty[i], 2 * kTile);
+      mbar_init(&sm.s_empty[i], kTile);          // the group that reads the buffer
     }
     sm.abort_flag = 0;
     fence_barrier_init();
@@ -225,7 +226,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     __syncwarp();
   } else {
-    const int wg = warp >> 2;                 // column half of every step
+    const int wg = warp >> 2;                 // takes the steps whose running number has this parity
     const int key = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float sc2 = a.scale * kLog2e;
@@ -260,24 +261,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * 2 * (int64_t)c + (int64_t)wg * c;
       const int nq = it.nq;
       const int steps = nkt * nq;
-      // The TMEM load of step s+1 is issued before the exponentials of step s, so that its latency
-      // (and the wait for the MMAs) hides behind them: two register sets, used alternately.
-      uint32_t ra[64], rb[64];
-      auto fetch = [&](int s, uint32_t* r) {      // issues the loads of step s; the caller waits for them
-        const int buf = (sg + s) & (kScoreBufs - 1);
-        ok = mbar_wait(&sm.s_full[buf], ((sg + s) / kScoreBufs) & 1, abort_flag, a.status, kTimeoutScore);
-        if (!ok) return;
-        tc_fence_after();
-        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64, r);
-        tmem_ld32(tmem + lane_base + buf * kTile + wg * 64 + 32, r + 32);
+      double total = 0.0;
+      int jacc = -1;     // key tile `total` belongs to
+      // stores this group's share of key tiles jacc .. upto - 1 (zero where it had no step)
+      auto flush = [&](int upto) {
+        for (int j = jacc < 0 ? 0 : jacc; j < upto; ++j) {
+          if (j * kTile + key < c) dst[j * kTile + key] = (j == jacc) ? (float)total : 0.f;
+        }
+        total = 0.0;
       };
-      auto landed = [&](int s) {                  // the values of step s are in registers: its buffer can be refilled
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&sm.s_empty[(sg + s) & (kScoreBufs - 1)]);
-      };
-      auto weigh = [&](const uint32_t* r, int qt) -> float {
-        const float4* bias4 = reinterpret_cast<const float4*>(&bias[qt * kTile + wg * 64]);
+      auto weigh = [&](const uint32_t* r, const float* bias_cols) -> float {
+        const float4* bias4 = reinterpret_cast<const float4*>(bias_cols);
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c4 = 0; c4 < 16; ++c4) {
@@ -289,30 +283,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         return (part[0] + part[1]) + (part[2] + part[3]);
       };
-      double total = 0.0;
-      int j = 0, qt = 0;
-      auto account = [&](float v) {               // adds step (j, qt); after a key tile's last query tile, stores
-        total += (double)v;
-        if (++qt == nq) {
-          if (j * kTile + key < c) dst[j * kTile + key] = (float)total;
-          total = 0.0; qt = 0; ++j;
+      for (int s = ((sg & 1) == wg) ? 0 : 1; s < steps && ok; s += 2) {
+        const int j = s / nq, qt = s - j * nq;
+        if (j != jacc) {
+          flush(j);
+          jacc = j;
         }
-      };
-      fetch(0, ra);
-      if (ok) landed(0);
-      for (int s = 0; s < steps && ok; s += 2) {
-        if (s + 1 < steps) fetch(s + 1, rb);
+        const int buf = (sg + s) & (kScoreBufs - 1);
+        ok = mbar_wait(&sm.s_full[buf], ((sg + s) / kScoreBufs) & 1, abort_flag, a.status, kTimeoutScore);
         if (!ok) break;
-        const float va = weigh(ra, qt);
-        if (s + 1 < steps) landed(s + 1);
-        account(va);
-        if (s + 1 >= steps) break;
-        if (s + 2 < steps) fetch(s + 2, ra);
-        if (!ok) break;
-        const float vb = weigh(rb, qt);
-        if (s + 2 < steps) landed(s + 2);
-        account(vb);
+        tc_fence_after();
+        uint32_t r[64];
+        const uint32_t t_addr = tmem + lane_base + buf * kTile;
+        tmem_ld32(t_addr, r);
+        tmem_ld32(t_addr + 32, r + 32);
+        tmem_wait_ld();
+        const float va = weigh(r, &bias[qt * kTile]);
+        tmem_ld32(t_addr + 64, r);
+        tmem_ld32(t_addr + 96, r + 32);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&sm.s_empty[buf]);            // the values are in registers: the buffer can be refilled
+        const float vb = weigh(r, &bias[qt * kTile + 64]);
+        total += (double)(va + vb);
       }
+      if (ok) flush(nkt);
       sg += steps;
     }
   }

@@ -270,16 +270,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         total = 0.0;
       };
-      auto weigh = [&](const uint32_t* r, const float* bias_cols) -> float {
+      // The 64 biases of a half step are fetched from shared memory before the wait for the TMEM
+      // load (the asm barrier keeps them there): inside the loop each load's latency would sit in
+      // front of its four exponentials, and two warps per scheduler cannot hide that.
+      auto fetch_bias = [&](float4* bv, const float* bias_cols) {
         const float4* bias4 = reinterpret_cast<const float4*>(bias_cols);
+#pragma unroll
+        for (int c4 = 0; c4 < 16; ++c4) bv[c4] = bias4[c4];
+      };
+      auto weigh = [&](const uint32_t* r, const float4* bv) -> float {
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c4 = 0; c4 < 16; ++c4) {
-          const float4 bv = bias4[c4];
-          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
-          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
-          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
-          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
+          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv[c4].x));
+          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv[c4].y));
+          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv[c4].z));
+          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv[c4].w));
         }
         return (part[0] + part[1]) + (part[2] + part[3]);
       };
@@ -295,16 +301,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tc_fence_after();
         uint32_t r[64];
         const uint32_t t_addr = tmem + lane_base + buf * kTile;
+        float4 bv[16];
         tmem_ld32(t_addr, r);
         tmem_ld32(t_addr + 32, r + 32);
+        fetch_bias(bv, &bias[qt * kTile]);
         tmem_wait_ld();
-        const float va = weigh(r, &bias[qt * kTile]);
+        const float va = weigh(r, bv);
         tmem_ld32(t_addr + 64, r);
         tmem_ld32(t_addr + 96, r + 32);
+        fetch_bias(bv, &bias[qt * kTile + 64]);
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(&sm.s_empty[buf]);            // the values are in registers: the buffer can be refilled
-        const float vb = weigh(r, &bias[qt * kTile + 64]);
+        const float vb = weigh(r, bv);
         total += (double)(va + vb);
       }
       if (ok) flush(nkt);

@@ -85,15 +85,18 @@ enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 // stream through once, 128 per tile. The grid is one CTA per SM; a CTA takes
 // items blockIdx.x, blockIdx.x + gridDim.x, ... so the K ring keeps running
 // from one item into the next: one lane of warp 9 issues the TMA loads. Per
-// (key tile, query tile) step one lane of warp 8 issues
-// S^T = K_tile . Q_tile^T (keys on the TMEM lane axis) into one of four TMEM
-// buffers. Warps 0-3 take the even steps, warps 4-7 the odd ones (so the two
+// (key tile, query tile) step S^T = K_tile . Q_tile^T (keys on the TMEM lane
+// axis) goes into one of four TMEM buffers; one lane of warp 8 issues the even
+// steps and one lane of warp 10 the odd ones, because the waits, fences and
+// commits around a step's eight MMAs cost an issuing thread almost as much time
+// as the MMAs take and the pipe idles meanwhile (measured: 1450 clocks per step
+// with one issuing thread against 512 of tensor work). Warps 0-3 take the even steps, warps 4-7 the odd ones (so the two
 // warps that share a scheduler are never in the same phase and the
 // special-function unit stays busy); a thread owns one key and sums
 // w_i * exp(s_ij - lse_i) over the 128 query columns of its steps, then writes
 // the key's partial score of (head, query chunk, step parity). A second kernel
 // adds the partial scores of a selection group in a fixed order.
-constexpr int kScoreThreads = 320;
+constexpr int kScoreThreads = 352;          // warps 0-7 compute, 8 and 10 issue MMAs, 9 loads
 constexpr int kScoreBufs = 4;              // TMEM buffers of 128 columns
 constexpr int kMaxQTiles = 4;              // query tiles resident per item
 constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
@@ -138,10 +141,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
-    mbar_init(&sm.q_empty, 1);
+    mbar_init(&sm.q_empty, 2);                   // both issuing threads
     for (int i = 0; i < kScoreTiles; ++i) {
       mbar_init(&sm.k_full[i], 1);
-      mbar_init(&sm.k_empty[i], 1);
+      mbar_init(&sm.k_empty[i], 2);
     }
     for (int i = 0; i < kScoreBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
@@ -190,9 +193,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == 8) {
-    // ---------------------------------------------------------------- MMA issue
+  } else if (warp == 8 || warp == 10) {
+    // ---------------------------------------------------------------- MMA issue: steps of one parity
     if (lane == 0 && my_items > 0) {
+      const int mine = warp == 8 ? 0 : 1;
       constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
       bool ok = true;
       int s = 0;                 // step = (key tile, query tile), numbered across items
@@ -200,10 +204,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       for (int k = 0; k < my_items && ok; ++k) {
         const ScoreItem it = item_of(k);
         ok = mbar_wait(&sm.q_full, k & 1, abort_flag, a.status, kTimeoutScore);
+        bool any_in_item = false;
         for (int j = 0; j < nkt && ok; ++j) {
           ok = mbar_wait(&sm.k_full[st], use & 1, abort_flag, a.status, kTimeoutScore);
           const uint64_t kd = smem_desc_sw128(smem_u32(sm.tiles[nq_max + st]), 16, 1024);
+          bool any = false;
           for (int qt = 0; qt < it.nq && ok; ++qt, ++s) {
+            if ((s & 1) != mine) continue;
             const int buf = s & (kScoreBufs - 1);
             if (s >= kScoreBufs)
               ok = mbar_wait(&sm.s_empty[buf], ((s / kScoreBufs) - 1) & 1, abort_flag, a.status, kTimeoutScore);
@@ -217,11 +224,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               mma_ss(d_tmem, kd + off, qd + off, idesc, kk > 0);
             }
             mma_commit(&sm.s_full[buf]);
-            if (qt == it.nq - 1) mma_commit(&sm.k_empty[st]);
+            any = true;
           }
+          if (!ok) break;
+          // the stage is free when both threads are through with it: after its MMAs of this tile, or at once
+          if (any) mma_commit(&sm.k_empty[st]);
+          else mbar_arrive(&sm.k_empty[st]);
+          any_in_item |= any;
           if (++st == kst) { st = 0; ++use; }
         }
-        if (ok) mma_commit(&sm.q_empty);
+        if (ok) {
+          if (any_in_item) mma_commit(&sm.q_empty);
+          else mbar_arrive(&sm.q_empty);
+        }
       }
     }
     __syncwarp();
@@ -289,8 +304,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         return (part[0] + part[1]) + (part[2] + part[3]);
       };
-      for (int s = ((sg & 1) == wg) ? 0 : 1; s < steps && ok; s += 2) {
-        const int j = s / nq, qt = s - j * nq;
+      const int s0 = ((sg & 1) == wg) ? 0 : 1;
+      int j = s0 / nq, qt = s0 - j * nq;         // key tile and query tile of step s, kept without dividing again
+      for (int s = s0; s < steps && ok; s += 2, qt += 2) {
+        while (qt >= nq) { qt -= nq; ++j; }
         if (j != jacc) {
           flush(j);
           jacc = j;

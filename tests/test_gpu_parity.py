@@ -125,6 +125,7 @@ SHAPES = [
     ("bf16", 2, 1, 1, 128, 1, 1, 1, 0),            # a single token
     ("bf16", 2, 2, 2, 128, 1, 1100, 200, 333),     # several key tiles per query tile, ragged last pair
     ("bf16", 4, 1, 1, 128, 2, 1536, 256, 700),     # GQA, six full query-tile pairs
+    ("bf16", 2, 2, 2, 128, 1, 900, 640, 100),      # window of five query tiles: two score chunks, the second short
 ]
 
 

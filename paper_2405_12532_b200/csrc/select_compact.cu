@@ -189,28 +189,40 @@ __global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, i
   const int32_t* idx = a.idx + (int64_t)bg * a.n_out;
   const int rows_per_iter = (kRowThreads * kRowUnroll) / lanes;   // lanes <= kRowThreads
   const int t = threadIdx.x;
-  for (int r0 = 0; r0 < a.n_out; r0 += rows_per_iter) {
-    uint4 buf[kRowUnroll];
-    int dst_row[kRowUnroll], ln[kRowUnroll];
+  // Chunk i + 1 is read while chunk i is written: the sources of a later chunk lie above every
+  // destination of an earlier one, so only the reads and writes of the same chunk need the barrier.
+  uint4 buf[2][kRowUnroll];
+  int dst_row[2][kRowUnroll], ln[kRowUnroll];
+#pragma unroll
+  for (int u = 0; u < kRowUnroll; ++u) ln[u] = (u * kRowThreads + t) % lanes;
+  auto read_chunk = [&](int r0, uint4* bf, int* dr) {
 #pragma unroll
     for (int u = 0; u < kRowUnroll; ++u) {
-      const int e = u * kRowThreads + t;
-      const int rr = e / lanes;
-      ln[u] = e % lanes;
-      dst_row[u] = -1;
+      const int rr = (u * kRowThreads + t) / lanes;
+      dr[u] = -1;
       if (rr < rows_per_iter && r0 + rr < a.n_out) {
         const int src = idx[r0 + rr];
         if (src != r0 + rr) {             // rows already in place are not touched
-          dst_row[u] = r0 + rr;
-          buf[u] = *reinterpret_cast<const uint4*>(base + (int64_t)src * row_bytes + ln[u] * 16);
+          dr[u] = r0 + rr;
+          bf[u] = *reinterpret_cast<const uint4*>(base + (int64_t)src * row_bytes + ln[u] * 16);
         }
       }
     }
-    __syncthreads();
+  };
+  auto write_chunk = [&](const uint4* bf, const int* dr) {
 #pragma unroll
     for (int u = 0; u < kRowUnroll; ++u)
-      if (dst_row[u] >= 0)
-        *reinterpret_cast<uint4*>(base + (int64_t)dst_row[u] * row_bytes + ln[u] * 16) = buf[u];
+      if (dr[u] >= 0) *reinterpret_cast<uint4*>(base + (int64_t)dr[u] * row_bytes + ln[u] * 16) = bf[u];
+  };
+  read_chunk(0, buf[0], dst_row[0]);
+  __syncthreads();
+  for (int r0 = 0; r0 < a.n_out; r0 += 2 * rows_per_iter) {
+    if (r0 + rows_per_iter < a.n_out) read_chunk(r0 + rows_per_iter, buf[1], dst_row[1]);
+    write_chunk(buf[0], dst_row[0]);
+    __syncthreads();
+    if (r0 + rows_per_iter >= a.n_out) break;
+    if (r0 + 2 * rows_per_iter < a.n_out) read_chunk(r0 + 2 * rows_per_iter, buf[0], dst_row[0]);
+    write_chunk(buf[1], dst_row[1]);
     __syncthreads();
   }
 }

@@ -84,19 +84,22 @@ enum TimeoutCode { kTimeoutScore = PYR_ERR_TIMEOUT };
 // queries, which stay in shared memory while the context keys of the head
 // stream through once, 128 per tile. The grid is one CTA per SM; a CTA takes
 // items blockIdx.x, blockIdx.x + gridDim.x, ... so the K ring keeps running
-// from one item into the next: one lane of warp 9 issues the TMA loads. Per
-// (key tile, query tile) step S^T = K_tile . Q_tile^T (keys on the TMEM lane
-// axis) goes into one of four TMEM buffers; one lane of warp 8 issues the even
-// steps and one lane of warp 10 the odd ones, because the waits, fences and
-// commits around a step's eight MMAs cost an issuing thread almost as much time
-// as the MMAs take and the pipe idles meanwhile (measured: 1450 clocks per step
-// with one issuing thread against 512 of tensor work). Warps 0-3 take the even steps, warps 4-7 the odd ones (so the two
-// warps that share a scheduler are never in the same phase and the
-// special-function unit stays busy); a thread owns one key and sums
-// w_i * exp(s_ij - lse_i) over the 128 query columns of its steps, then writes
-// the key's partial score of (head, query chunk, step parity). A second kernel
-// adds the partial scores of a selection group in a fixed order.
-constexpr int kScoreThreads = 352;          // warps 0-7 compute, 8 and 10 issue MMAs, 9 loads
+// from one item into the next (one lane of a loader warp issues the TMA loads).
+// Per (key tile, query tile) step S^T = K_tile . Q_tile^T (keys on the TMEM lane
+// axis) goes into one of four TMEM buffers; one lane each of two warps issues
+// the even and the odd steps, because the waits, fences and commits around a
+// step's eight MMAs cost an issuing thread almost as much time as the MMAs take
+// and the pipe idles meanwhile (measured: 1450 clocks per step with one issuing
+// thread against 512 of tensor work). Sixteen compute warps in four groups:
+// group g takes the steps s with s % 4 == g (so the four warps that share a
+// scheduler are always in different phases and the special-function unit stays
+// busy); a thread owns one key and sums w_i * exp(s_ij - lse_i) over the 128
+// query columns of its steps, then writes the key's partial score of
+// (head, query chunk, group). A second kernel adds the partial scores of a
+// selection group in a fixed order.
+constexpr int kScoreGroups = 4;             // compute groups of four warps
+constexpr int kScoreCompute = 4 * kScoreGroups;
+constexpr int kScoreThreads = (kScoreCompute + 3) * 32;   // then: MMA issue (even steps), TMA loads, MMA issue (odd steps)
 constexpr int kScoreBufs = 4;              // TMEM buffers of 128 columns
 constexpr int kMaxQTiles = 4;              // query tiles resident per item
 constexpr int kScoreTiles = 6;             // 32 KB tiles of shared memory: the query tiles, then the K stages
@@ -153,7 +156,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     sm.abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 8) {
+  if (warp == kScoreCompute) {
     tmem_alloc(&sm.tmem_base, kScoreBufs * kTile);
     tmem_relinquish();
   }
@@ -162,7 +165,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp == 9) {
+  if (warp == kScoreCompute + 1) {
     // ---------------------------------------------------------------- TMA loads
     if (lane == 0 && my_items > 0) {
       prefetch_tensormap(&map_q);
@@ -193,10 +196,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == 8 || warp == 10) {
+  } else if (warp == kScoreCompute || warp == kScoreCompute + 2) {
     // ---------------------------------------------------------------- MMA issue: steps of one parity
     if (lane == 0 && my_items > 0) {
-      const int mine = warp == 8 ? 0 : 1;
+      const int mine = warp == kScoreCompute ? 0 : 1;
       constexpr uint32_t idesc = idesc_bf16(kTile, kTile, false, false);
       bool ok = true;
       int s = 0;                 // step = (key tile, query tile), numbered across items
@@ -241,7 +244,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     __syncwarp();
   } else {
-    const int wg = warp >> 2;                 // takes the steps whose running number has this parity
+    const int wg = warp >> 2;                 // takes the steps whose running number is wg modulo 4
     const int key = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const float sc2 = a.scale * kLog2e;
@@ -253,27 +256,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                  ? log2f(a.w[qi]) - a.lse[((int64_t)it.b * a.Hq + it.h) * n + c + qi] * kLog2e
                  : -INFINITY;
     };
-    float nb0 = 0.f, nb1 = 0.f;
-    if (my_items > 0) {
-      const ScoreItem it = item_of(0);
-      nb0 = bias_of(it, threadIdx.x);
-      nb1 = bias_of(it, threadIdx.x + 2 * kTile);
-    }
+    static_assert(kScoreGroups * kTile == kMaxQTiles * kTile, "one bias entry per compute thread");
+    float nb = my_items > 0 ? bias_of(item_of(0), threadIdx.x) : 0.f;
     bool ok = true;
     int sg = 0;   // steps of earlier items
     for (int k = 0; k < my_items && ok; ++k) {
       const ScoreItem it = item_of(k);
       float* bias = sm.bias[k & 1];
-      bias[threadIdx.x] = nb0;
-      bias[threadIdx.x + 2 * kTile] = nb1;
+      bias[threadIdx.x] = nb;
       // every thread is past its reads of this buffer (item k - 2) since it went through the barrier of item k - 1
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (k + 1 < my_items) {
-        const ScoreItem nx = item_of(k + 1);
-        nb0 = bias_of(nx, threadIdx.x);
-        nb1 = bias_of(nx, threadIdx.x + 2 * kTile);
-      }
-      float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * 2 * (int64_t)c + (int64_t)wg * c;
+      asm volatile("bar.sync 1, %0;" ::"n"(kScoreGroups * kTile) : "memory");
+      if (k + 1 < my_items) nb = bias_of(item_of(k + 1), threadIdx.x);
+      float* dst = partial + (((int64_t)it.b * a.Hq + it.h) * nchunk + it.chunk) * kScoreGroups * (int64_t)c + (int64_t)wg * c;
       const int nq = it.nq;
       const int steps = nkt * nq;
       double total = 0.0;
@@ -285,28 +279,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         total = 0.0;
       };
-      // The 64 biases of a half step are fetched from shared memory before the wait for the TMEM
-      // load (the asm barrier keeps them there): inside the loop each load's latency would sit in
-      // front of its four exponentials, and two warps per scheduler cannot hide that.
-      auto fetch_bias = [&](float4* bv, const float* bias_cols) {
+      // 32 query columns at a time: the TMEM load of the next quarter is in flight during the
+      // exponentials of this one (two register sets)
+      auto weigh = [&](const uint32_t* r, const float* bias_cols) -> float {
         const float4* bias4 = reinterpret_cast<const float4*>(bias_cols);
-#pragma unroll
-        for (int c4 = 0; c4 < 16; ++c4) bv[c4] = bias4[c4];
-      };
-      auto weigh = [&](const uint32_t* r, const float4* bv) -> float {
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c4 = 0; c4 < 16; ++c4) {
-          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv[c4].x));
-          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv[c4].y));
-          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv[c4].z));
-          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv[c4].w));
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 bv = bias4[c4];
+          part[0] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 0]), sc2, bv.x));
+          part[1] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 1]), sc2, bv.y));
+          part[2] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 2]), sc2, bv.z));
+          part[3] += ex2(fmaf(__uint_as_float(r[c4 * 4 + 3]), sc2, bv.w));
         }
         return (part[0] + part[1]) + (part[2] + part[3]);
       };
-      const int s0 = ((sg & 1) == wg) ? 0 : 1;
+      const int s0 = (wg - sg) & (kScoreGroups - 1);
       int j = s0 / nq, qt = s0 - j * nq;         // key tile and query tile of step s, kept without dividing again
-      for (int s = s0; s < steps && ok; s += 2, qt += 2) {
+      for (int s = s0; s < steps && ok; s += kScoreGroups, qt += kScoreGroups) {
         while (qt >= nq) { qt -= nq; ++j; }
         if (j != jacc) {
           flush(j);
@@ -316,22 +306,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         ok = mbar_wait(&sm.s_full[buf], ((sg + s) / kScoreBufs) & 1, abort_flag, a.status, kTimeoutScore);
         if (!ok) break;
         tc_fence_after();
-        uint32_t r[64];
         const uint32_t t_addr = tmem + lane_base + buf * kTile;
-        float4 bv[16];
-        tmem_ld32(t_addr, r);
-        tmem_ld32(t_addr + 32, r + 32);
-        fetch_bias(bv, &bias[qt * kTile]);
+        const float* bq = &bias[qt * kTile];
+        uint32_t ra[32], rb[32];
+        tmem_ld32(t_addr, ra);
         tmem_wait_ld();
-        const float va = weigh(r, bv);
-        tmem_ld32(t_addr + 64, r);
-        tmem_ld32(t_addr + 96, r + 32);
-        fetch_bias(bv, &bias[qt * kTile + 64]);
+        tmem_ld32(t_addr + 32, rb);
+        float v = weigh(ra, bq);
+        tmem_wait_ld();
+        tmem_ld32(t_addr + 64, ra);
+        v += weigh(rb, bq + 32);
+        tmem_wait_ld();
+        tmem_ld32(t_addr + 96, rb);
+        v += weigh(ra, bq + 64);
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(&sm.s_empty[buf]);            // the values are in registers: the buffer can be refilled
-        const float vb = weigh(r, bv);
-        total += (double)(va + vb);
+        v += weigh(rb, bq + 96);
+        total += (double)v;
       }
       if (ok) flush(nkt);
       sg += steps;
@@ -339,7 +331,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == kScoreCompute) {
     tc_fence_after();
     tmem_dealloc(tmem, kScoreBufs * kTile);
   }
@@ -364,6 +356,7 @@ bool score_tc_supported(const PrefillArgs& a) {
 }
 bool tensor_maps_available() { return encode_fn() != nullptr; }
 
+int score_tc_groups() { return kScoreGroups; }
 int score_tc_chunks(int L) { return ((L + kTile - 1) / kTile + kMaxQTiles - 1) / kMaxQTiles; }
 
 cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s) {
@@ -387,7 +380,7 @@ cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s
   if (e != cudaSuccess) return e;
   const int heads = a.Hq / a.G;
   dim3 rgrid((c + 255) / 256, a.G, a.B);
-  score_reduce_kernel<<<rgrid, 256, 0, s>>>(partial, a.score, c, a.G, heads * nchunk * 2, heads, a.status);
+  score_reduce_kernel<<<rgrid, 256, 0, s>>>(partial, a.score, c, a.G, heads * nchunk * kScoreGroups, heads, a.status);
   return cudaGetLastError();
 }
 

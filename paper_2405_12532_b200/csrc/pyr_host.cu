@@ -71,7 +71,7 @@ void plan(const pyr_config_t* c, Layout* lay) {
   // per-head partial scores of the tensor-core score kernel (bf16, head_dim 128 only)
   lay->score_part = off;
   if (c->dtype == PYR_BF16 && D == 128 && c0 > 0)
-    off = align_up(off + B * Hq * (size_t)pyr::score_tc_chunks(L) * 2 * (size_t)c0 * 4, kAlign);
+    off = align_up(off + B * Hq * (size_t)pyr::score_tc_chunks(L) * pyr::score_tc_groups() * (size_t)c0 * 4, kAlign);
   lay->lse = off;    off = align_up(off + B * Hq * (size_t)N * 4, kAlign);
   lay->idx = off;    off = align_up(off + B * G * (size_t)N * 4, kAlign);
   lay->pos0 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);

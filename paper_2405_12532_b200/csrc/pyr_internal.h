@@ -78,9 +78,10 @@ inline void decode_split_rule(int batch, int n_kv_heads, int total, int* splits_
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s);     // bf16, D = 128, tcgen05
-// `partial` holds B * Hq * score_tc_chunks(L) * 2 * c floats: per-head partial scores, summed by a second kernel
+// `partial` holds B * Hq * score_tc_chunks(L) * score_tc_groups() * c floats: per-head partial scores, summed by a second kernel
 cudaError_t launch_score_tc(const PrefillArgs& a, float* partial, cudaStream_t s);
 int score_tc_chunks(int L);
+int score_tc_groups();
 bool prefill_tc_supported(const PrefillArgs& a);
 bool score_tc_supported(const PrefillArgs& a);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);

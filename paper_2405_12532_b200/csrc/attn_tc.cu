@@ -51,6 +51,7 @@ struct AttnSmem {
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2], p_ready[2], o_done[2];         // per tile
   uint64_t stage_free;                               // the stores of one epilogue have read o_stage
+  uint64_t turn[2];                                  // [tile]: that tile may run its exponentials (8 warp arrivals)
   float xch[2][2][kTile];                            // [tile][key half][row]: row maximum / row sum of one half
   uint32_t tmem_base;
   int abort_flag;
@@ -125,6 +126,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.o_done[i], 1);
     }
     mbar_init(&sm.stage_free, 1);
+    mbar_init(&sm.turn[0], 8);
+    mbar_init(&sm.turn[1], 8);
     sm.abort_flag = 0;
     fence_barrier_init();
   }
@@ -275,6 +278,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     int nb = 0;                  // blocks this tile has finished
     int ep_base = 0;             // epilogues of earlier blocks (they use the staging tile in a fixed order)
     bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
+    // The two tiles take turns at the exponentials (tile 0 first), so that one tile's special-function
+    // work runs while the other tile's MMAs do, instead of both tiles doing the same thing at once.
+    int turns = 0;               // turns taken so far (the same number on both tiles)
     for (int it = 0; ok; ++it) {
       Block bk;
       if (!block_at(it, part, parts, n, &bk)) break;
@@ -283,6 +289,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ep_base += 1;
         continue;
       }
+      const int shared_steps = bk.nkt1 ? bk.nkt0 : 0;    // steps that both tiles have in this block
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
       float m_used = -INFINITY, l = 0.f;                 // l: this thread's share of the row sum
       for (int t = 0; t < nkt_w && ok; ++t) {
@@ -336,6 +343,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         if (need) m_used = mrow;
         const float neg_m = -m_used;
+        const bool take_turn = t < shared_steps;
+        if (take_turn && (w == 1 || turns > 0)) {
+          ok = mbar_wait(&sm.turn[w], (w ? turns : turns - 1) & 1, abort_flag, a.status, code);
+          if (!ok) break;
+        }
         // pass 2: P = exp2(s * scale - m) in bf16, 32 columns at a time; P of columns c .. c + 31
         // lands on TMEM columns c / 2 .. of this thread's half (already read)
         float part[4] = {0.f, 0.f, 0.f, 0.f};
@@ -360,6 +372,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             p[c2] = pack_bf16(p0, p1);
           }
           tmem_st16(my_s + ch * 16, p);
+        }
+        if (take_turn) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.turn[w ^ 1]);
+          ++turns;
         }
         tmem_wait_st();
         tc_fence_before();

@@ -38,7 +38,7 @@ constexpr int kTile = 128;                  // query rows per tile, keys per K/V
 constexpr int kHalf = 64;                   // keys per half-step
 constexpr int kHalfBytes = kTile * 128;     // one [128 rows x 64 bf16] swizzled half tile (half of D)
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128 x 128] bf16 tile = two halves along D
-constexpr int kSoftmaxWarps = 16;          // two tiles x two key halves x four TMEM lane quarters
+constexpr int kSoftmaxWarps = 8;
 constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
 constexpr float kRescaleStep = 8.0f;
 
@@ -49,15 +49,11 @@ struct AttnSmem {
   alignas(1024) uint8_t o_stage[kTileBytes];         // a [128 x 128] bf16 tile of O on its way out (both tiles use it)
   uint64_t q_full[2], q_empty[2];                    // per tile
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
-  uint64_t s_full[2], p_ready[2], o_done[2];         // per tile
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
   uint64_t stage_free;                               // the stores of one epilogue have read o_stage
-  uint64_t turn[2];                                  // [tile]: that tile may run its exponentials (8 warp arrivals)
-  float xch[2][2][kTile];                            // [tile][key half][row]: row maximum / row sum of one half
   uint32_t tmem_base;
   int abort_flag;
 };
-
-static_assert(sizeof(AttnSmem) <= 232448, "AttnSmem must fit the 227 KB a CTA can opt in to");
 
 // Geometry of one block of the head: two consecutive 128-row tiles that share their K/V tiles.
 // The tiles are paired from the last one down, so that with an odd number of tiles the block that
@@ -97,14 +93,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                PrefillArgs a, int parts) {
-  // The tiles need 1024-byte alignment (128-byte swizzle) and the struct fills the shared memory a CTA
-  // can have, so there is no room to align by hand: a misaligned base is reported, not worked around.
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  AttnSmem& sm = *reinterpret_cast<AttnSmem*>(smem_raw);
-  if ((smem_u32(smem_raw) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicCAS(a.status, 0, PYR_ERR_UNSUPPORTED);
-    return;
-  }
+  extern __shared__ uint8_t smem_raw[];
+  AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int h = blockIdx.x / parts, part = blockIdx.x % parts, b = blockIdx.y;
   const int g = h / (a.Hq / a.Hkv);
@@ -121,13 +111,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.k_empty[i], 2);
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 2);
-      mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.p_ready[i], 2 * kTile);
-      mbar_init(&sm.o_done[i], 1);
+      for (int bf = 0; bf < 2; ++bf) {
+        mbar_init(&sm.s_full[i][bf], 1);
+        mbar_init(&sm.p_ready[i][bf], kTile);
+        mbar_init(&sm.o_done[i][bf], 1);
+      }
     }
     mbar_init(&sm.stage_free, 1);
-    mbar_init(&sm.turn[0], 8);
-    mbar_init(&sm.turn[1], 8);
     sm.abort_flag = 0;
     fence_barrier_init();
   }
@@ -187,22 +177,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---------------------------------------------------------------- MMA issue, one thread per tile
     const int w = warp - kSoftmaxWarps;
     if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // S = Q K^T (128 keys), both K-major
+      constexpr uint32_t idesc_s = idesc_bf16(kTile, kHalf, false, false);   // S = Q K^T (64 keys), both K-major
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // O += P V, V is MN-major
       // operand descriptors are built once; a k-step only adds a constant to the start-address field
       const uint64_t dq = smem_desc_sw128(smem_u32(sm.q[w]), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
       const uint64_t dv0 = smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
-      const uint32_t s_tmem = tmem + w * 256, o_tmem = s_tmem + 128;
+      const uint32_t t_base = tmem + w * 256, o_tmem = t_base + 128;
       bool ok = true;
       int kvu = 0;   // K/V tiles of the ring that earlier blocks used
       int nq = 0;    // Q loads of this tile consumed
-      int cnt = 0;   // key tiles of this tile done in earlier blocks
+      int hs = 0;    // half-steps of this tile done in earlier blocks (even)
       for (int it = 0; ok; ++it) {
         Block bk;
         if (!block_at(it, part, parts, n, &bk)) break;
         const int nkt_w = w ? bk.nkt1 : bk.nkt0;
+        const int T = 2 * nkt_w;
         // when the key tiles come in descending order, the one tile 0 does not read comes first
         const int skip = ((it & 1) && nkt_w && nkt_w < bk.nkt) ? 1 : 0;
         // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
@@ -214,7 +205,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (ok) ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
           if (ok) mbar_arrive(&sm.v_empty[st]);
         };
-        if (nkt_w == 0) {
+        // S(t): keys 64 t .. 64 t + 63 = rows (t & 1) * 64 .. of K tile t / 2, into S buffer t & 1
+        auto issue_s = [&](int t) {
+          const int ring = kvu + skip + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) {
+            ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+            if (!ok) return;
+            tc_fence_after();
+          }
+          const uint64_t kd = (st ? dk1 : dk0) + (uint64_t)((bf * kHalf * 128) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
+            mma_ss(t_base + bf * kHalf, dq + off, kd + off, idesc_s, kk > 0);
+          }
+          mma_commit(&sm.s_full[w][bf]);
+          if (bf == 1) mma_commit(&sm.k_empty[st]);
+          if (t == T - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
+        };
+        if (T == 0) {
           for (int j = 0; j < bk.nkt && ok; ++j) release(kvu + j);
           kvu += bk.nkt;
           continue;
@@ -222,116 +231,93 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (skip) release(kvu);
         if (ok) ok = mbar_wait(&sm.q_full[w], nq & 1, abort_flag, a.status, code);
         ++nq;
-        for (int j = 0; j < nkt_w && ok; ++j) {
-          const int ring = kvu + skip + j, st = ring & 1, par = (ring >> 1) & 1;
-          ok = mbar_wait(&sm.k_full[st], par, abort_flag, a.status, code);
+        if (ok) issue_s(0);
+        if (ok) issue_s(1);
+        for (int t = 0; t < T && ok; ++t) {
+          const int ring = kvu + skip + (t >> 1), st = ring & 1, bf = t & 1;
+          if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
+          if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
-          // S(j) lands on the columns that held S(j-1) and P(j-1): the pipe runs it after PV(j-1)
-          const uint64_t kd = st ? dk1 : dk0;
+          const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-            mma_ss(s_tmem, dq + off, kd + off, idesc_s, kk > 0);
-          }
-          mma_commit(&sm.s_full[w]);
-          mma_commit(&sm.k_empty[st]);
-          if (j == nkt_w - 1) mma_commit(&sm.q_empty[w]);     // last read of this block's Q tile
-          ok = mbar_wait(&sm.v_full[st], par, abort_flag, a.status, code);
-          if (ok) ok = mbar_wait(&sm.p_ready[w], (cnt + j) & 1, abort_flag, a.status, code);
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t vd = st ? dv1 : dv0;
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)   // 16 keys per step: 8 TMEM columns of P (keys 64.. start at column 64), 16 rows of V
-            mma_ts(o_tmem, s_tmem + (kk >> 2) * kHalf + (kk & 3) * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
-                   (j > 0 || kk > 0) ? 1u : 0u);
-          if (j == nkt_w - 1) mma_commit(&sm.o_done[w]);      // one phase per block: the epilogue waits for it
-          mma_commit(&sm.v_empty[st]);
+          for (int kk = 0; kk < 4; ++kk)   // 16 keys per step: 8 TMEM columns of P, 16 rows of V
+            mma_ts(o_tmem, t_base + bf * kHalf + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+                   (t > 0 || kk > 0) ? 1u : 0u);
+          if (t >= T - 2) mma_commit(&sm.o_done[w][bf]);   // the block's last two PVs: one phase per block each
+          if (bf == 1) mma_commit(&sm.v_empty[st]);
+          if (t + 2 < T) issue_s(t + 2);
         }
         if (ok && nkt_w < bk.nkt && !skip) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
         kvu += bk.nkt;
-        cnt += nkt_w;
+        hs += T;
       }
     }
     __syncwarp();
   } else {
-    // ---------------------------------------------------------------- softmax, two threads per query row
-    // Warps 0-7 serve tile 0, warps 8-15 tile 1. Inside a tile, warp & 3 picks the 32 TMEM lanes
-    // (rows) and (warp >> 2) & 1 the half of a 128-key S tile: the two threads of a row (same lane,
-    // warps p and p + 4 of the tile) each own 64 key columns, agree on the row maximum through
-    // shared memory, and each keep their share of the row sum.
-    const int w = warp >> 3;
-    const int half = (warp >> 2) & 1;
-    const int row = (warp & 3) * 32 + lane;
+    // ---------------------------------------------------------------- softmax, thread = query row
+    const int w = warp >> 2;
+    const int row = threadIdx.x & (kTile - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t s_base = tmem + lane_base + w * 256;   // S: 128 fp32 columns
-    const uint32_t my_s = s_base + half * kHalf;          // this thread's 64 S columns; its P lands on the first 32
-    const uint32_t o_addr = s_base + 128 + half * kHalf;  // this thread's 64 O columns
+    const uint32_t t_base = tmem + lane_base + w * 256;
+    const uint32_t o_addr = t_base + 128;
     const float sc2 = a.scale * kLog2e;
-    const int pair_bar = 1 + w * 4 + (warp & 3);          // named barrier of the two warps that share these rows
-    float* xch_mine = &sm.xch[w][half][row];
-    const float* xch_other = &sm.xch[w][half ^ 1][row];
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory"); };
     bool ok = true;
-    int cnt = 0;                 // key tiles of this tile done in earlier blocks
+    int hs = 0;    // half-steps of this tile done in earlier blocks (even)
     int nb = 0;                  // blocks this tile has finished
-    int ep_base = 0;             // epilogues of earlier blocks (they use the staging tile in a fixed order)
+    int ep_base = 0;             // epilogues of earlier blocks
     bool release_due = false;    // (thread 0 of the tile) its stores may still be reading the staging tile
-    // The two tiles take turns at the exponentials (tile 0 first), so that one tile's special-function
-    // work runs while the other tile's MMAs do, instead of both tiles doing the same thing at once.
-    int turns = 0;               // turns taken so far (the same number on both tiles)
     for (int it = 0; ok; ++it) {
       Block bk;
       if (!block_at(it, part, parts, n, &bk)) break;
-      const int nkt_w = w ? bk.nkt1 : bk.nkt0;
-      if (nkt_w == 0) {
+      const int T = 2 * (w ? bk.nkt1 : bk.nkt0);
+      if (T == 0) {
         ep_base += 1;
         continue;
       }
-      const int shared_steps = bk.nkt1 ? bk.nkt0 : 0;    // steps that both tiles have in this block
       const int i = bk.r0 + w * kTile + row;             // query row of this thread
-      float m_used = -INFINITY, l = 0.f;                 // l: this thread's share of the row sum
-      for (int t = 0; t < nkt_w && ok; ++t) {
-        // key tile of this step: ascending order in even blocks, descending in odd ones
-        const int kt = (it & 1) ? nkt_w - 1 - t : t;
-        const bool diag = kt == nkt_w - 1;
-        const int key0 = kt * kTile + half * kHalf;        // first key of this thread's columns
-        ok = mbar_wait(&sm.s_full[w], (cnt + t) & 1, abort_flag, a.status, code);
+      float m_used = -INFINITY, l = 0.f;
+      for (int t = 0; t < T && ok; ++t) {
+        const int bf = t & 1;
+        const uint32_t s_addr = t_base + bf * kHalf;
+        ok = mbar_wait(&sm.s_full[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
         tc_fence_after();
-        // pass 1: maximum of this thread's 64 columns, 32 at a time
-        float mx = -INFINITY;
+        uint32_t s[64];
+        tmem_ld32(s_addr, s);
+        tmem_ld32(s_addr + 32, s + 32);
+        tmem_wait_ld();
+        // key tile of this half-step: they come in ascending order in even blocks, descending in odd ones
+        const int kt = (it & 1) ? (T >> 1) - 1 - (t >> 1) : (t >> 1);
+        if (kt == (T >> 1) - 1) {         // inside the diagonal key tile: key 128 kt + 64 (t & 1) + col is visible iff col <= lim
+          const int lim = i - (kt * kTile + (t & 1) * kHalf);
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t s[32];
-          tmem_ld32(my_s + ch * 32, s);
-          tmem_wait_ld();
-          if (diag) {
-            const int lim = i - (key0 + ch * 32);          // column col is visible iff col <= lim
-#pragma unroll
-            for (int col = 0; col < 32; ++col)
-              if (col > lim) s[col] = 0xff800000u;         // -inf
-          }
-          float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-          for (int col = 0; col < 32; col += 4) {
-            m0 = max3(m0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
-            m1 = max3(m1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
-          }
-          mx = fmaxf(mx, fmaxf(m0, m1));
+          for (int col = 0; col < 64; ++col)
+            if (col > lim) s[col] = 0xff800000u;   // -inf
         }
-        *xch_mine = mx;
-        pair_sync();
-        const float mrow = fmaxf(mx, *xch_other) * sc2;    // (-inf when the row sees none of the 128 keys)
-        pair_sync();                                       // the slot may be written again
-        const bool need = mrow > m_used + kRescaleStep;    // also true on the first step (m_used = -inf)
-        if (t > 0 && __any_sync(0xffffffffu, need)) {
-          // O holds every PV up to PV(t-1): S(t) was issued after it and the pipe runs in order.
-          // Each thread rescales its own 64 columns of O; both threads of a row take the same decision.
-          const float f = need ? ex2(m_used - mrow) : 1.f;
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
+        for (int col = 0; col < 64; col += 8) {
+          mx0 = max3(mx0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
+          mx1 = max3(mx1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
+          mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
+          mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
+        }
+        // (-inf when every key of this half-step is hidden from the row: then nothing changes and P = 0)
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;
+        const bool need = mx > m_used + kRescaleStep;      // also true on the first half-step (m_used = -inf)
+        if (t > 0 && __any_sync(0xffffffffu, need)) {
+          // O may be rescaled once it holds every PV up to PV(t-1), the last one these threads have
+          // fed. The issuing thread runs S(t+1) right after PV(t-1) and the pipe keeps that order,
+          // so S(t+1) having landed is the signal (its barrier is one phase ahead of what this
+          // thread has consumed, so the parity wait is valid); the block's last PVs have their own.
+          if (t + 1 < T) ok = mbar_wait(&sm.s_full[w][(t + 1) & 1], ((hs + t + 1) >> 1) & 1, abort_flag, a.status, code);
+          else ok = mbar_wait(&sm.o_done[w][0], nb & 1, abort_flag, a.status, code);
+          if (!ok) break;
+          tc_fence_after();
+          const float f = need ? ex2(m_used - mx) : 1.f;
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
             uint32_t o[32];
             tmem_ld32(o_addr + ch * 32, o);
             tmem_wait_ld();
@@ -341,46 +327,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
           l *= f;
         }
-        if (need) m_used = mrow;
+        if (need) m_used = mx;
         const float neg_m = -m_used;
-        const bool take_turn = t < shared_steps;
-        if (take_turn && (w == 1 || turns > 0)) {
-          ok = mbar_wait(&sm.turn[w], (w ? turns : turns - 1) & 1, abort_flag, a.status, code);
-          if (!ok) break;
-        }
-        // pass 2: P = exp2(s * scale - m) in bf16, 32 columns at a time; P of columns c .. c + 31
-        // lands on TMEM columns c / 2 .. of this thread's half (already read)
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
-          uint32_t s[32];
-          tmem_ld32(my_s + ch * 32, s);
-          tmem_wait_ld();
-          if (diag) {
-            const int lim = i - (key0 + ch * 32);
-#pragma unroll
-            for (int col = 0; col < 32; ++col)
-              if (col > lim) s[col] = 0xff800000u;
-          }
           uint32_t p[16];
 #pragma unroll
           for (int c2 = 0; c2 < 16; ++c2) {
-            const float p0 = ex2(fmaf(__uint_as_float(s[2 * c2]), sc2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(s[2 * c2 + 1]), sc2, neg_m));
+            const float p0 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2]), sc2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(s[ch * 32 + 2 * c2 + 1]), sc2, neg_m));
             part[c2 & 1] += p0;
             part[2 + (c2 & 1)] += p1;
             p[c2] = pack_bf16(p0, p1);
           }
-          tmem_st16(my_s + ch * 16, p);
-        }
-        if (take_turn) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.turn[w ^ 1]);
-          ++turns;
+          tmem_st16(s_addr + ch * 16, p);
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&sm.p_ready[w]);
+        mbar_arrive(&sm.p_ready[w][bf]);
         l += (part[0] + part[1]) + (part[2] + part[3]);
         if (release_due) {       // only ever set in thread 0 of the tile
           bulk_wait_read_all();
@@ -390,43 +355,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       // epilogue of the block; the next block's first PV cannot start before these threads have
       // delivered its P(0), i.e. after they are done reading O here
-      if (ok) ok = mbar_wait(&sm.o_done[w], nb & 1, abort_flag, a.status, code);
+      if (ok) ok = mbar_wait(&sm.o_done[w][1], nb & 1, abort_flag, a.status, code);
       if (!ok) break;
       tc_fence_after();
-      *xch_mine = l;
-      pair_sync();
-      const float l_row = l + *xch_other;
-      pair_sync();
-      if (half == 0 && i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l_row)) * kLn2;
-      // O leaves through shared memory and two TMA stores (rows past n are clipped by the store);
-      // each thread stages its 64 columns. The epilogue before this one (the other tile's, or this
-      // tile's of the previous block when that block had one tile) must have been read out first.
-      const float inv = 1.f / l_row;
+      // O leaves through shared memory and two TMA stores (rows past n are clipped by the store).
+      // The epilogue before this one (the other tile's, or this tile's of the previous block when
+      // that block had one tile) must have been read out of the staging tile first.
+      if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_used + log2f(l)) * kLn2;
+      const float inv = 1.f / l;
       const int seq = ep_base + w;
       if (seq > 0) {
         ok = mbar_wait(&sm.stage_free, (seq - 1) & 1, abort_flag, a.status, code);
         if (!ok) break;
       }
-      uint8_t* my_row = sm.o_stage + half * kHalfBytes + row * 128;
+      uint8_t* my_row = sm.o_stage + row * 128;
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t o[32];
-        tmem_ld32(o_addr + ch * 32, o);
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t o[64];
+        tmem_ld32(o_addr + hf * 64, o);
+        tmem_ld32(o_addr + hf * 64 + 32, o + 32);
         tmem_wait_ld();
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {       // 16-byte chunk c of the row sits at c ^ (row & 7): the 128-byte swizzle
+        for (int ch = 0; ch < 8; ++ch) {     // 16-byte chunk ch of the row sits at ch ^ (row & 7): the 128-byte swizzle
           uint4 pk;
-          pk.x = pack_bf16(__uint_as_float(o[q4 * 8 + 0]) * inv, __uint_as_float(o[q4 * 8 + 1]) * inv);
-          pk.y = pack_bf16(__uint_as_float(o[q4 * 8 + 2]) * inv, __uint_as_float(o[q4 * 8 + 3]) * inv);
-          pk.z = pack_bf16(__uint_as_float(o[q4 * 8 + 4]) * inv, __uint_as_float(o[q4 * 8 + 5]) * inv);
-          pk.w = pack_bf16(__uint_as_float(o[q4 * 8 + 6]) * inv, __uint_as_float(o[q4 * 8 + 7]) * inv);
-          *reinterpret_cast<uint4*>(my_row + (((ch * 4 + q4) ^ (row & 7)) << 4)) = pk;
+          pk.x = pack_bf16(__uint_as_float(o[ch * 8 + 0]) * inv, __uint_as_float(o[ch * 8 + 1]) * inv);
+          pk.y = pack_bf16(__uint_as_float(o[ch * 8 + 2]) * inv, __uint_as_float(o[ch * 8 + 3]) * inv);
+          pk.z = pack_bf16(__uint_as_float(o[ch * 8 + 4]) * inv, __uint_as_float(o[ch * 8 + 5]) * inv);
+          pk.w = pack_bf16(__uint_as_float(o[ch * 8 + 6]) * inv, __uint_as_float(o[ch * 8 + 7]) * inv);
+          *reinterpret_cast<uint4*>(my_row + hf * kHalfBytes + ((ch ^ (row & 7)) << 4)) = pk;
         }
       }
       fence_proxy_async();
-      if (w == 0) asm volatile("bar.sync 9, 256;" ::: "memory");   // the 256 threads of this tile
-      else asm volatile("bar.sync 10, 256;" ::: "memory");
-      if (row == 0 && half == 0) {
+      if (w == 0) asm volatile("bar.sync 1, 128;" ::: "memory");   // the 128 threads of this tile
+      else asm volatile("bar.sync 2, 128;" ::: "memory");
+      if (row == 0) {
         tma_store_4d(&map_o, sm.o_stage, 0, h, bk.r0 + w * kTile, b);
         tma_store_4d(&map_o, sm.o_stage + kHalfBytes, 64, h, bk.r0 + w * kTile, b);
         bulk_commit();
@@ -437,7 +399,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           release_due = true; // signalled a little later, off the path to the next block's first P
         }
       }
-      cnt += nkt_w;
+      hs += T;
       ++nb;
       ep_base += bk.nkt1 ? 2 : 1;
     }
@@ -445,7 +407,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bulk_wait_read_all();
       mbar_arrive(&sm.stage_free);
     }
-    if (row == 0 && half == 0) bulk_wait_all();   // the last stores have left shared memory and are complete
+    if (row == 0) bulk_wait_all();   // the last stores have left shared memory and are complete
   }
   tc_fence_before();
   __syncthreads();
@@ -468,7 +430,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
       !make_tensor_map_bf16(&mk, a.k, a.B, a.n, a.Hkv, a.D, a.ksb, a.ksn, a.ksh, kTile) ||
       !make_tensor_map_bf16(&mv, a.v, a.B, a.n, a.Hkv, a.D, a.ksb, a.ksn, a.ksh, kTile))
     return cudaErrorInvalidValue;
-  const size_t smem = sizeof(AttnSmem);
+  const size_t smem = sizeof(AttnSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   // One CTA per (sequence, head) when that fills the SMs evenly; otherwise deal each head's blocks

@@ -51,7 +51,6 @@ struct AttnSmem {
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage; empty = both issuing threads arrived
   uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];   // [tile][S buffer]
   uint64_t stage_free;                               // the stores of one epilogue have read o_stage
-  uint64_t batch_turn[2];                            // [tile]: that tile's issuing thread may issue its next PV + S batch
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -119,8 +118,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     mbar_init(&sm.stage_free, 1);
-    mbar_init(&sm.batch_turn[0], 1);
-    mbar_init(&sm.batch_turn[1], 1);
     sm.abort_flag = 0;
     fence_barrier_init();
   }
@@ -192,17 +189,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int kvu = 0;   // K/V tiles of the ring that earlier blocks used
       int nq = 0;    // Q loads of this tile consumed
       int hs = 0;    // half-steps of this tile done in earlier blocks (even)
-      // The two issuing threads take turns with their PV(t) + S(t+2) batches (tile 0 first) on the
-      // half-steps both tiles have. Left alone, both tiles become ready together, their batches
-      // interleave in the pipe and both S groups arrive late; in turns one tile's S is early and the
-      // tiles settle half a step apart.
-      int turns = 0;
       for (int it = 0; ok; ++it) {
         Block bk;
         if (!block_at(it, part, parts, n, &bk)) break;
         const int nkt_w = w ? bk.nkt1 : bk.nkt0;
         const int T = 2 * nkt_w;
-        const int shared_steps = bk.nkt1 ? 2 * bk.nkt0 : 0;
         // when the key tiles come in descending order, the one tile 0 does not read comes first
         const int skip = ((it & 1) && nkt_w && nkt_w < bk.nkt) ? 1 : 0;
         // K/V tile `ring` of the CTA's load sequence is not read by this tile: wait until it has
@@ -246,9 +237,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const int ring = kvu + skip + (t >> 1), st = ring & 1, bf = t & 1;
           if (bf == 0) ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
           if (ok) ok = mbar_wait(&sm.p_ready[w][bf], ((hs + t) >> 1) & 1, abort_flag, a.status, code);
-          const bool take_turn = t < shared_steps;
-          if (ok && take_turn && (w == 1 || turns > 0))
-            ok = mbar_wait(&sm.batch_turn[w], (w ? turns : turns - 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = (st ? dv1 : dv0) + (uint64_t)((bf * kHalf * 128) >> 4);
@@ -259,10 +247,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (t >= T - 2) mma_commit(&sm.o_done[w][bf]);   // the block's last two PVs: one phase per block each
           if (bf == 1) mma_commit(&sm.v_empty[st]);
           if (t + 2 < T) issue_s(t + 2);
-          if (take_turn) {
-            mbar_arrive(&sm.batch_turn[w ^ 1]);
-            ++turns;
-          }
         }
         if (ok && nkt_w < bk.nkt && !skip) release(kvu + bk.nkt - 1);   // tile 1's diagonal K/V tile
         kvu += bk.nkt;

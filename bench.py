@@ -32,7 +32,7 @@ from paper_2405_12532_b200 import synth
 
 METRIC = "prefill tokens/s + decode tokens/s at 7B shapes 64x2k"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch divided by its algorithmic bytes
-# (542.47 MB / 537.13 MB in profiles/decode_kernel_7b_2k_batch16.txt). Set to None when the kernel changes.
+# (542.04 MB / 537.13 MB in profiles/decode_kernel_7b_2k_batch16.txt). Set to None when the kernel changes.
 DECODE_TRAFFIC_RATIO = 542.04 / 537.13
 DEFAULT_WORKLOAD = "7b_64x2k"
 

@@ -1,11 +1,14 @@
 // tcgen05 causal attention of the prefill step (bf16, head_dim 128):
 // Algorithm 1, "compute attention weights of KV", and the attention output.
 //
-// A CTA owns one (sequence, head) and walks its query rows in blocks of 256:
-// two 128-row tiles that share every K and V tile the CTA loads (TMA, 128 keys
-// per tile, two stages each). Because the CTA stays on the head, the loads, the
-// first MMAs and the output epilogue of consecutive blocks overlap instead of
-// paying a prologue per block, and every CTA of the grid does the same work.
+// A CTA owns one (sequence, head), or one of 2, 4 or 8 equal shares of it when
+// there are too few heads to fill the SMs evenly, and walks its query rows in
+// blocks of 256: two 128-row tiles that share every K and V tile the CTA loads
+// (TMA, 128 keys per tile, two stages each; up through the key tiles in even
+// blocks and down in odd ones, so that a block starts on tiles still in L2).
+// Because the CTA stays on the head, the loads, the first MMAs and the output
+// epilogue (a staged tile and two TMA stores) of consecutive blocks overlap
+// instead of paying a prologue per block, and every CTA does the same work.
 //   warps 0-3 / 4-7   softmax of tile 0 / 1, thread = one query row
 //   warp 8 / 9        MMA issue for tile 0 / 1 (one lane each)
 //   warp 10           TMA loads (one lane)

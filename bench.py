@@ -365,7 +365,16 @@ def oracle_sample(workload: str, layers=None):
     ratio = synth.ratio_schedule(w)
     budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
     nL = len(budgets)
-    layers = layers or sorted({0, nL // 2, nL - 1})
+    if layers is None:
+        # evenly spaced layers, as many (3 to 12) as keep the sample near 10-15 s of host time:
+        # about 8e9 head x key x query x dim products per second on the hosts measured so far
+        cost = lambda ls: sum(budgets[l]["n_in"] ** 2 for l in ls) * w["n_q_heads"] * w["head_dim"]
+        spaced = lambda k: sorted({round(i * (nL - 1) / (k - 1)) for i in range(k)})
+        layers = spaced(min(3, nL)) if nL > 1 else [0]
+        for k in range(4, min(nL, 12) + 1):
+            if cost(spaced(k)) > 1.0e11:
+                break
+            layers = spaced(k)
     cores = len(os.sched_getaffinity(0))
     torch.set_num_threads(cores)
     t_total = 0.0

@@ -30,6 +30,19 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _check_register_split(ptxas_log: str) -> None:
+    """The attention kernel moves registers between its warpgroups (setmaxnreg) and sizes the split
+    for 168 registers per thread at launch (kRegsLaunch in csrc/attn_tc.cu). If ptxas ever allocates
+    fewer, the softmax warps would wait for registers that do not exist: refuse to build that."""
+    import re
+    m = re.search(r"attn_tc_kernel.*?Used (\d+) registers", ptxas_log, re.S)
+    if not m:
+        raise RuntimeError("ptxas log has no register count for attn_tc_kernel")
+    if int(m.group(1)) != 168:
+        raise RuntimeError(f"attn_tc_kernel launches with {m.group(1)} registers per thread, not the 168 its "
+                           "setmaxnreg split (kRegsLaunch) assumes: adjust kRegsLaunch / kRegsSoftmax in csrc/attn_tc.cu")
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
@@ -52,6 +65,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
     with open(os.path.join(objdir, "ptxas.log"), "w") as f:
         f.write("\n".join(log))
+    _check_register_split("\n".join(log))
     if verbose:
         print("\n".join(log))
     cmd = [nvcc, "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]

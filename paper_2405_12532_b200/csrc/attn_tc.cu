@@ -488,6 +488,10 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+  // the register split inside the kernel is sized for kRegsLaunch registers per thread at launch
+  cudaFuncAttributes fa;
+  if ((e = cudaFuncGetAttributes(&fa, attn_tc_kernel)) != cudaSuccess) return e;
+  if (fa.numRegs != kRegsLaunch) return cudaErrorInvalidConfiguration;
   size_t smem = kSmemNeed + 1024;
   if (smem > (size_t)smem_max) smem = (size_t)smem_max;
   if (smem < kSmemNeed) return cudaErrorInvalidConfiguration;

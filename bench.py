@@ -366,13 +366,13 @@ def oracle_sample(workload: str, layers=None):
     budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
     nL = len(budgets)
     if layers is None:
-        # evenly spaced layers, as many (3 to 12) as keep the sample near 10-15 s of host time:
+        # evenly spaced layers, as many (3 to 16) as keep the sample near 10-15 s of host time:
         # about 8e9 head x key x query x dim products per second on the hosts measured so far
         cost = lambda ls: sum(budgets[l]["n_in"] ** 2 for l in ls) * w["n_q_heads"] * w["head_dim"]
         spaced = lambda k: sorted({round(i * (nL - 1) / (k - 1)) for i in range(k)})
         layers = spaced(min(3, nL)) if nL > 1 else [0]
-        for k in range(4, min(nL, 12) + 1):
-            if cost(spaced(k)) > 1.0e11:
+        for k in range(4, min(nL, 16) + 1):
+            if cost(spaced(k)) > 1.3e11:
                 break
             layers = spaced(k)
     cores = len(os.sched_getaffinity(0))

@@ -164,9 +164,10 @@ def test_budget_matches_workload_tables(row):
     assert ks[-len(last):] == last
     for l, x in enumerate(b):
         assert x["n_out"] == x["k"] + L
-        assert x["k"] == min(x["c"], int(np.floor(ratio[l] * (N - L))))
+        assert x["k"] <= x["c"] == x["n_in"] - L
         if l:
             assert x["n_in"] == b[l - 1]["n_out"]
+            assert x["k"] <= b[l - 1]["k"]                   # the pyramid never widens
 
 
 def test_budget_edges():
@@ -244,6 +245,51 @@ def test_prefill_layer_structure_and_ratio_one():
     one = oracle.prefill_layer(Q, K, V, L, 13, 1)
     assert one["kept"].shape == (B, 1, 13 + L)
     np.testing.assert_allclose(one["score"][:, 0], half["score"].mean(1), rtol=1e-13)
+
+
+def _heads_by_loops(Q, K, L, w, scale, b):
+    """Per-head scores of sequence b by explicit loops; query head h reads KV
+    head h // (Hq / Hkv), written out here independently of the oracle."""
+    Hq, Hkv = Q.shape[2], K.shape[2]
+    per_kv = Hq // Hkv
+    return np.stack([_score_by_loops(Q[b, :, h], K[b, :, h // per_kv], L, w, scale) for h in range(Hq)])
+
+
+@pytest.mark.parametrize("G", [2, 1])
+def test_prefill_layer_score_grouped_heads_by_loops(G):
+    # Hq = 8 query heads over Hkv = 2 KV heads: a wrong head-to-KV-head mapping (h % Hkv in place
+    # of h // r), a wrong pooling axis or a missing mean changes the pooled score
+    B, n, Hq, Hkv, D, L = 2, 21, 8, 2, 4, 5
+    Q, K, V = _rand(B, n, Hq, D), _rand(B, n, Hkv, D), _rand(B, n, Hkv, D)
+    w = oracle.recent_weights(L)
+    scale = 0.6
+    got = oracle.prefill_layer(Q, K, V, L, 7, G, scale=scale)["score"]
+    assert got.shape == (B, G, n - L)
+    for b in range(B):
+        E = _heads_by_loops(Q, K, L, w, scale, b)                      # [Hq, c]
+        per = Hq // G
+        for g in range(G):
+            want = sum(E[g * per + i] for i in range(per)) / per
+            np.testing.assert_allclose(got[b, g], want, rtol=1e-12)
+
+
+def test_default_softmax_scale_is_inverse_sqrt_head_dim():
+    assert oracle.softmax_scale_default(64) == 0.125
+    assert abs(oracle.softmax_scale_default(128) - 0.08838834764831845) < 1e-16     # 2^-3.5
+    assert oracle.softmax_scale_default(16) == 0.25
+    # the defaults of the layer and of the decode step against the library's own default scale
+    B, n, H, D, L = 1, 24, 2, 16, 4
+    Q, K, V = _rand(B, n, H, D), _rand(B, n, H, D), _rand(B, n, H, D)
+    out = oracle.prefill_layer(Q, K, V, L, 5, H)
+    t = lambda x: torch.from_numpy(x[0]).permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V), is_causal=True)[0]
+    np.testing.assert_allclose(out["O"][0], ref.permute(1, 0, 2).numpy(), rtol=1e-10, atol=1e-12)
+    w = oracle.recent_weights(L)
+    for h in range(H):
+        np.testing.assert_allclose(out["score"][0, h], _score_by_loops(Q[0, :, h], K[0, :, h], L, w, 0.25), rtol=1e-12)
+    dec, _, _ = oracle.decode_attention(Q[0, n - 1], K[0, : n - 1].transpose(1, 0, 2), V[0, : n - 1].transpose(1, 0, 2),
+                                        K[0, n - 1], V[0, n - 1])
+    np.testing.assert_allclose(dec, ref[:, n - 1].numpy(), rtol=1e-10, atol=1e-12)
 
 
 def test_nesting_of_positions_across_layers():

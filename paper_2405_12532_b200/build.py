@@ -32,15 +32,20 @@ def needs_build() -> bool:
 
 def _check_register_split(ptxas_log: str) -> None:
     """The attention kernel moves registers between its warpgroups (setmaxnreg) and sizes the split
-    for 168 registers per thread at launch (kRegsLaunch in csrc/attn_tc.cu). If ptxas ever allocates
-    fewer, the softmax warps would wait for registers that do not exist: refuse to build that."""
+    for kRegsLaunch registers per thread at launch (csrc/attn_tc.cu). If ptxas ever allocates fewer,
+    the softmax warps would wait for registers that do not exist: refuse to build that. Spills in
+    that kernel mean the split no longer fits the code: refuse those too."""
     import re
-    m = re.search(r"attn_tc_kernel.*?Used (\d+) registers", ptxas_log, re.S)
+    with open(os.path.join(CSRC, "attn_tc.cu")) as f:
+        want = int(re.search(r"kRegsLaunch\s*=\s*(\d+)", f.read()).group(1))
+    m = re.search(r"attn_tc_kernel.*?(\d+) bytes spill stores.*?Used (\d+) registers", ptxas_log, re.S)
     if not m:
         raise RuntimeError("ptxas log has no register count for attn_tc_kernel")
-    if int(m.group(1)) != 168:
-        raise RuntimeError(f"attn_tc_kernel launches with {m.group(1)} registers per thread, not the 168 its "
-                           "setmaxnreg split (kRegsLaunch) assumes: adjust kRegsLaunch / kRegsSoftmax in csrc/attn_tc.cu")
+    if int(m.group(2)) != want:
+        raise RuntimeError(f"attn_tc_kernel launches with {m.group(2)} registers per thread, not the {want} its "
+                           "setmaxnreg split (kRegsLaunch) assumes: adjust the split in csrc/attn_tc.cu")
+    if int(m.group(1)) != 0:
+        raise RuntimeError(f"attn_tc_kernel spills {m.group(1)} bytes: its register split no longer fits the code")
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

@@ -6,28 +6,26 @@
 // one at a time, longest first (key tiles up in even tiles of the walk and down
 // in odd ones, so that a tile starts on K/V still in L2). The K tiles of all
 // query tiles form one stream r = 0, 1, 2, ... that every role walks on its own.
-//   warps 0-3   softmax group 0, thread = one query row
-//   warps 4-7   softmax group 1 (same rows), and the epilogue of every tile
-//   warp 8      issues the S MMAs:  S(r) = Q K(r)^T, 128 keys, Q and K from shared memory
-//   warp 9      TMA loads of Q and K (two stages of K)
-//   warp 10     issues the PV MMAs: O += P(r) V(r), P from tensor memory
-//   warp 11     TMA loads of V (two stages; a V stage is freed up to three K tiles after the
-//               K stage, so the K loads must not queue behind the V loads)
-// Tensor memory (512 columns): three S buffers of 128 fp32 columns (K tile r uses
-// buffer r % 3; P as bf16 overwrites the first 64 columns) and O (128 columns).
-// S(r) may be issued as soon as PV(r - 3) has read its P, so the S MMAs run up to
-// three K tiles ahead of the softmax and never wait for it; separate issuing
-// threads keep either kind of MMA from queueing behind the other's waits.
-// Within a query tile the two softmax groups take alternate K tiles, counted
-// from the tile's end, so group 1 always has the last one and writes the tile
-// out. A thread holds its row's 128 scores in registers (the four issuing and
-// loading warps hand their registers to the softmax warps at the start). What
-// couples the groups is the maximum used in the exponent: the thread of K tile
-// r reads the value published for r - 1, raises it only when the row maximum
+//   warps 0-3    softmax group 0, thread = one query row; takes the even r
+//   warps 4-7    softmax group 1 (same rows); takes the odd r
+//   warp 8       issues the S MMAs:  S(r) = Q K(r)^T, 128 keys, Q and K from shared memory
+//   warp 9       TMA loads of Q and K (two stages of K)
+//   warp 10      issues the PV MMAs: O += P(r) V(r), P from tensor memory
+//   warp 11      TMA loads of V (two stages)
+//   warps 12-15  epilogue of every tile: O / row sum -> bf16 -> shared memory -> TMA store, and lse
+// Tensor memory (512 columns): S buffers 0 and 1 (128 fp32 columns each), P
+// buffers 0 and 1 (64 columns each: 128 bf16), O (128 columns). Group g owns S
+// buffer g, P buffer g and their barriers. A softmax thread reads its row's 128
+// scores into registers and releases the S buffer at once, so S(r + 2) is
+// computed while the exponentials of r are taken; P(r) is written to the P
+// buffer once PV(r - 2) has read it. What couples the groups is the maximum
+// used in the exponent: the thread of K tile r reads the value published for
+// r - 1 (one word per row and tile parity), raises it only when the row maximum
 // has grown by more than 2^8 (which keeps rescaling of O, a TMEM round trip,
 // rare), and publishes its own before it starts on the exponentials. Each group
-// keeps its own row sum; the epilogue adds them under the final maximum, so
-// the result is the exact softmax.
+// keeps its own row sum and hands it, with the maximum it is relative to, to the
+// epilogue warps, which add the two under the final maximum: the result is the
+// exact softmax. The softmax groups never wait for a tile to be written out.
 //
 // All mbarriers live across tiles, so every role counts the phases it has
 // consumed (a parity wait is only valid one phase behind the barrier; the
@@ -49,22 +47,26 @@ constexpr int kTile = 128;                  // query rows per tile, keys per K/V
 constexpr int kHalfBytes = kTile * 128;     // one [128 rows x 64 bf16] swizzled half tile (half of D)
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128 x 128] bf16 tile = two halves along D
 constexpr int kSoftmaxWarps = 8;
-constexpr int kThreads = (kSoftmaxWarps + 4) * 32;
+constexpr int kWarpS = 8, kWarpLoadQK = 9, kWarpPV = 10, kWarpLoadV = 11, kWarpEpi = 12;
+constexpr int kThreads = 16 * 32;
 constexpr float kRescaleStep = 8.0f;
-constexpr int kRegsLaunch = 168, kRegsSoftmax = 232, kRegsIssue = 40;   // kRegsLaunch must be what ptxas reports for the kernel
-constexpr int kSBufs = 3;                   // S buffers of 128 fp32 columns: TMEM columns 0..383
+// kRegsLaunch must be what ptxas reports for the kernel
+constexpr int kRegsLaunch = 128, kRegsSoftmax = 208, kRegsIssue = 40, kRegsEpi = 56;
+constexpr uint32_t kColP = 256;             // P buffers: columns 256..319 and 320..383
 constexpr uint32_t kColO = 384;             // O: columns 384..511
+constexpr int kFinSlots = 4;                // tiles whose row sums may be waiting for the epilogue
 
 struct AttnSmem {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[2][kTileBytes];
   alignas(1024) uint8_t v[2][kTileBytes];
-  alignas(1024) uint8_t o_stage[kTileBytes];         // a [128 x 128] bf16 tile of O on its way out
-  unsigned long long m_slot[kTile];                  // per row: (K tiles decided so far) << 32 | bits of the maximum in use
-  float l_even[2][kTile];                            // [tile parity][row]: group 0's row sum of the tile
+  alignas(1024) uint8_t o_stage[kHalfBytes];         // a [128 x 64] bf16 half tile of O on its way out
+  unsigned long long m_slot[2][kTile];               // [tile parity][row]: (K tiles decided so far) << 32 | bits of the maximum in use
+  unsigned long long fin[2][kFinSlots][kTile];                   // [group][tile % 4][row]: bits of the group's row sum of the tile << 32 | bits of the maximum it is relative to
   uint64_t q_full[2], q_empty[2];                    // per Q buffer
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];   // per stage
-  uint64_t s_full[3], p_ready[3], pv_done[3];        // per S buffer (K tile r of the stream uses buffer r % 3): S landed / P written / PV has read P
+  uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2];   // per group: S landed / S is in registers / P written / PV has read P
+  uint64_t o_full;                                   // the last PV of a tile is complete
   uint64_t o_free;                                   // the epilogue has read O
   uint32_t tmem_base;
   int abort_flag;
@@ -105,14 +107,25 @@ __device__ __forceinline__ bool slot_wait(const volatile unsigned long long* slo
   return false;
 }
 
+// Barrier of the 128 threads of one role that also tells every one of them whether any came with `bad`.
+template <int kId>
+__device__ __forceinline__ bool bar_any(bool bad) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(any) : "r"((uint32_t)(bad ? 1 : 0)), "n"(kId) : "memory");
+  return any != 0;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
                 PrefillArgs a, int parts) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // The tiles need 1024-byte alignment. The launch asks for what the struct needs plus as much of
-  // a kilobyte as the SM's limit leaves; if the window's base is not aligned well enough for that,
-  // the CTA reports it instead of running past the end.
+  // The tiles need 1024-byte alignment. The launch asks for what the struct needs plus a kilobyte;
+  // if the window's base is not aligned well enough for that, the CTA reports it instead of
+  // running past the end.
   const uint32_t pad = (1024u - (smem_u32(smem_raw) & 1023u)) & 1023u;
   uint32_t dyn_bytes;
   asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
@@ -127,7 +140,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = a.n;
   volatile int* abort_flag = &sm.abort_flag;
-  if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -137,18 +149,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.k_empty[i], 1);
       mbar_init(&sm.v_full[i], 1);
       mbar_init(&sm.v_empty[i], 1);
-    }
-    for (int i = 0; i < kSBufs; ++i) {
       mbar_init(&sm.s_full[i], 1);
+      mbar_init(&sm.s_free[i], kTile);
       mbar_init(&sm.p_ready[i], kTile);
       mbar_init(&sm.pv_done[i], 1);
     }
+    mbar_init(&sm.o_full, 1);
     mbar_init(&sm.o_free, kTile);
-    sm.abort_flag = 0;
+    // an earlier CTA of this launch gave up: the whole CTA leaves together (decided by one thread)
+    sm.abort_flag = *reinterpret_cast<volatile int*>(a.status) != 0 ? 2 : 0;
     fence_barrier_init();
   }
-  if (threadIdx.x < kTile) sm.m_slot[threadIdx.x] = 0ull;
-  if (warp == kSoftmaxWarps) {
+  if (threadIdx.x < 2 * kTile) (&sm.m_slot[0][0])[threadIdx.x] = 0ull;
+  __syncthreads();
+  if (sm.abort_flag == 2) return;
+  if (warp == kWarpS) {
     tmem_alloc(&sm.tmem_base, 512);
     tmem_relinquish();
   }
@@ -157,14 +172,79 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const int code = PYR_ERR_TIMEOUT;
-  // Register split: the block starts with kThreads x kRegsLaunch registers; the four issuing /
-  // loading warps (one warpgroup) give theirs up, the two softmax warpgroups take them:
-  // 256 x kRegsSoftmax + 128 x kRegsIssue <= kThreads x kRegsLaunch.
-  static_assert(256 * kRegsSoftmax + 128 * kRegsIssue <= kThreads * kRegsLaunch, "register split exceeds the launch's total");
+  // Register split: the block starts with kThreads x kRegsLaunch registers; the issuing / loading
+  // warps and the epilogue warps (one warpgroup each) give registers up, the two softmax
+  // warpgroups take them.
+  static_assert(256 * kRegsSoftmax + 128 * kRegsIssue + 128 * kRegsEpi <= kThreads * kRegsLaunch,
+                "register split exceeds the launch's total");
 
-  if (warp >= kSoftmaxWarps) {
+  if (warp >= kWarpEpi) {
+    // ---------------------------------------------------------------- epilogue of every tile
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsEpi));
+    const int row = threadIdx.x & (kTile - 1);
+    const uint32_t o_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kColO;
+    uint8_t* my_row = sm.o_stage + row * 128;
+    bool ok = true, stored = false;
+    int ring0 = 0;
+    for (int it = 0;; ++it) {
+      Tile tl;
+      if (!tile_at(it, part, parts, n, &tl)) break;
+      const int nkt = tl.nkt;
+      const int i = tl.r0 + row;
+      const int gf = (ring0 + nkt - 1) & 1;               // the group that took the tile's last K tile
+      if (ok) ok = mbar_wait(&sm.o_full, it & 1, abort_flag, a.status, code);
+      if (bar_any<1>(!ok)) break;
+      tc_fence_after();
+      // Row sums of both groups, each relative to the maximum in use when the group left the tile;
+      // the last K tile's maximum is the final one. (Written before the groups' arrivals for their
+      // last P of the tile, which the tile's last PV follows.)
+      const unsigned long long f = *reinterpret_cast<volatile unsigned long long*>(&sm.fin[gf][it & (kFinSlots - 1)][row]);
+      float l = __uint_as_float((uint32_t)(f >> 32));
+      const float m_fin = __uint_as_float((uint32_t)f);
+      if (nkt >= 2) {
+        const unsigned long long o2 = *reinterpret_cast<volatile unsigned long long*>(&sm.fin[gf ^ 1][it & (kFinSlots - 1)][row]);
+        l += __uint_as_float((uint32_t)(o2 >> 32)) * ex2(__uint_as_float((uint32_t)o2) - m_fin);
+      }
+      if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_fin + log2f(l)) * kLn2;
+      const float inv = 1.f / l;
+      // O leaves through shared memory, one [128 x 64] half at a time (rows past n are clipped by the store)
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        if (row == 0 && stored) bulk_wait_read_all();      // the store before has read the staging half
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+        for (int c32 = 0; c32 < 2; ++c32) {
+          uint32_t o[32];
+          tmem_ld32(o_addr + hf * 64 + c32 * 32, o);
+          tmem_wait_ld();
+          if (hf == 1 && c32 == 1) {           // the accumulator is in registers: the next tile may overwrite it
+            tc_fence_before();
+            mbar_arrive(&sm.o_free);
+          }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {     // 16-byte chunk c of the half row sits at c ^ (row & 7): the 128-byte swizzle
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(o[ch * 8 + 0]) * inv, __uint_as_float(o[ch * 8 + 1]) * inv);
+            pk.y = pack_bf16(__uint_as_float(o[ch * 8 + 2]) * inv, __uint_as_float(o[ch * 8 + 3]) * inv);
+            pk.z = pack_bf16(__uint_as_float(o[ch * 8 + 4]) * inv, __uint_as_float(o[ch * 8 + 5]) * inv);
+            pk.w = pack_bf16(__uint_as_float(o[ch * 8 + 6]) * inv, __uint_as_float(o[ch * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(my_row + (((c32 * 4 + ch) ^ (row & 7)) << 4)) = pk;
+          }
+        }
+        fence_proxy_async();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (row == 0) {
+          tma_store_4d(&map_o, sm.o_stage, hf * 64, h, tl.r0, b);
+          bulk_commit();
+          stored = true;
+        }
+      }
+      ring0 += nkt;
+    }
+    if (row == 0 && stored) bulk_wait_all();   // the last stores have left shared memory and are complete
+  } else if (warp >= kSoftmaxWarps) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
-  if (warp == kSoftmaxWarps + 1) {
+  if (warp == kWarpLoadQK) {
     // ---------------------------------------------------------------- TMA loads of Q and K
     if (lane == 0) {
       prefetch_tensormap(&map_q);
@@ -205,10 +285,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == kSoftmaxWarps + 3) {
+  } else if (warp == kWarpLoadV) {
     // ---------------------------------------------------------------- TMA loads of V
-    // (a thread of their own: a V stage is released by its PV, up to three K tiles after the S
-    // MMAs released the K stage, and the K loads must not wait for that)
+    // (a thread of their own: a V stage is released by its PV, later than the S MMAs release
+    // the K stage, and the K loads must not wait for that)
     if (lane == 0) {
       prefetch_tensormap(&map_v);
       bool ok = true;
@@ -229,14 +309,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == kSoftmaxWarps) {
+  } else if (warp == kWarpS) {
     // ---------------------------------------------------------------- S MMAs: S(r) = Q K^T for K tile r of the stream
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_bf16(kTile, kTile, false, false);   // both K-major
       const uint64_t dq0 = smem_desc_sw128(smem_u32(sm.q[0]), 16, 1024), dq1 = smem_desc_sw128(smem_u32(sm.q[1]), 16, 1024);
       const uint64_t dk0 = smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024), dk1 = smem_desc_sw128(smem_u32(sm.k[1]), 16, 1024);
       bool ok = true;
-      int ring = 0, sb = 0, sph = 0;                   // K tiles so far; S buffer ring % 3 and the parity of ring / 3
+      int ring = 0;                                    // K tiles so far; buffer and stage ring & 1, phase (ring >> 1) & 1
       for (int it = 0; ok; ++it) {
         Tile tl;
         if (!tile_at(it, part, parts, n, &tl)) break;
@@ -244,27 +324,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         ok = mbar_wait(&sm.q_full[bq], (it >> 1) & 1, abort_flag, a.status, code);
         const uint64_t dq = bq ? dq1 : dq0;
         for (int j = 0; j < tl.nkt && ok; ++j, ++ring) {
-          const int st = ring & 1;
-          ok = mbar_wait(&sm.k_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
-          // the buffer is free once PV(ring - 3) has read its P
-          if (ok && ring >= kSBufs) ok = mbar_wait(&sm.pv_done[sb], sph ^ 1, abort_flag, a.status, code);
+          const int st = ring & 1, ph = (ring >> 1) & 1;
+          ok = mbar_wait(&sm.k_full[st], ph, abort_flag, a.status, code);
+          // the buffer is free once the softmax threads of K tile ring - 2 hold its scores in registers
+          if (ok && ring >= 2) ok = mbar_wait(&sm.s_free[st], ph ^ 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
           const uint64_t kd = st ? dk1 : dk0;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
             const uint64_t off = (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4);
-            mma_ss(tmem + sb * kTile, dq + off, kd + off, idesc_s, kk > 0);
+            mma_ss(tmem + st * kTile, dq + off, kd + off, idesc_s, kk > 0);
           }
-          mma_commit(&sm.s_full[sb]);
+          mma_commit(&sm.s_full[st]);
           mma_commit(&sm.k_empty[st]);
           if (j == tl.nkt - 1) mma_commit(&sm.q_empty[bq]);     // last read of this Q tile
-          if (++sb == kSBufs) { sb = 0; sph ^= 1; }
         }
       }
     }
     __syncwarp();
-  } else if (warp == kSoftmaxWarps + 2) {
+  } else if (warp == kWarpPV) {
     // ---------------------------------------------------------------- PV MMAs: O += P(r) V
     if (lane == 0) {
       constexpr uint32_t idesc_o = idesc_bf16(kTile, kTile, false, true);    // V is MN-major
@@ -272,26 +351,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint64_t dv1 = smem_desc_sw128(smem_u32(sm.v[1]), kHalfBytes, 1024);
       const uint32_t o_tmem = tmem + kColO;
       bool ok = true;
-      int ring = 0, sb = 0, sph = 0;
+      int ring = 0;
       for (int it = 0; ok; ++it) {
         Tile tl;
         if (!tile_at(it, part, parts, n, &tl)) break;
         // the first PV of a tile overwrites the accumulator of the tile before it
         if (it >= 1) ok = mbar_wait(&sm.o_free, (it - 1) & 1, abort_flag, a.status, code);
         for (int j = 0; j < tl.nkt && ok; ++j, ++ring) {
-          const int st = ring & 1;
-          ok = mbar_wait(&sm.v_full[st], (ring >> 1) & 1, abort_flag, a.status, code);
-          if (ok) ok = mbar_wait(&sm.p_ready[sb], sph, abort_flag, a.status, code);
+          const int st = ring & 1, ph = (ring >> 1) & 1;
+          ok = mbar_wait(&sm.v_full[st], ph, abort_flag, a.status, code);
+          if (ok) ok = mbar_wait(&sm.p_ready[st], ph, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
           const uint64_t vd = st ? dv1 : dv0;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)   // 16 keys per MMA: 8 TMEM columns of P, 16 rows of V
-            mma_ts(o_tmem, tmem + sb * kTile + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
+            mma_ts(o_tmem, tmem + kColP + st * 64 + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o,
                    (j > 0 || kk > 0) ? 1u : 0u);
-          mma_commit(&sm.pv_done[sb]);
+          mma_commit(&sm.pv_done[st]);
           mma_commit(&sm.v_empty[st]);
-          if (++sb == kSBufs) { sb = 0; sph ^= 1; }
+          if (j == tl.nkt - 1) mma_commit(&sm.o_full);           // the tile's accumulator is complete
         }
       }
     }
@@ -300,11 +379,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else {
     // ---------------------------------------------------------------- softmax, thread = query row
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    const int grp = warp >> 2;                           // 1: takes every tile's last K tile, and the epilogue
+    const int grp = warp >> 2;                           // takes the K tiles r of the stream with r % 2 == grp
     const int row = threadIdx.x & (kTile - 1);
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_base = tmem + lane_base;
+    const uint32_t t_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t o_addr = t_base + kColO;
+    const uint32_t s_addr = t_base + grp * kTile;
+    const uint32_t p_addr = t_base + kColP + grp * 64;
     const float sc2 = a.scale * kLog2e;
     bool ok = true;
     int ring0 = 0;               // K tiles of earlier tiles
@@ -316,56 +396,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int i = tl.r0 + row;                          // query row of this thread
       const int tp = it & 1;
       float m_mine = -INFINITY, l = 0.f;                  // this group's row sum and the maximum it is relative to
-      float m_other = -INFINITY;                          // (group 1) the maximum group 0's row sum is relative to
-      // The groups alternate within the tile, counted from its end: group 1 has the last K tile.
-      for (int j = (((nkt - 1) & 1) == grp) ? 1 : 0; j < nkt && ok; j += 2) {
+      // The groups alternate along the whole stream, so the group that finishes a tile is never the
+      // one that the next tile starts with.
+      const int j0 = ((ring0 & 1) == grp) ? 0 : 1;
+      const int j_last = ((ring0 + nkt - 1) & 1) == grp ? nkt - 1 : nkt - 2;   // this group's last K tile of the tile
+      for (int j = j0; j < nkt && ok; j += 2) {
         const int ring = ring0 + j;
-        const int sb = ring % kSBufs, sph = (ring / kSBufs) & 1;
-        const uint32_t s_addr = t_base + sb * kTile;
-        ok = mbar_wait(&sm.s_full[sb], sph, abort_flag, a.status, code);
+        const int ph = (ring >> 1) & 1;
+        ok = mbar_wait(&sm.s_full[grp], ph, abort_flag, a.status, code);
         if (!ok) break;
         tc_fence_after();
+        uint32_t s[kTile];               // the row's 128 scores (the softmax warps hold the registers for it)
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, s + ch * 32);
+        // While the scores are on their way: the maximum in use after the K tile before this one,
+        // from the partner thread of this row. A tile's first K tile starts from -inf and waits for
+        // nobody: the word of this tile parity was last read two tiles ago (see the P-buffer wait).
+        float m_prev = -INFINITY;
+        if (j > 0) ok = slot_wait(&sm.m_slot[tp][row], (uint32_t)ring, &m_prev, abort_flag, a.status, code);
         // key tile of this step: ascending in even tiles of the walk, descending in odd ones
         const int kt = (it & 1) ? nkt - 1 - j : j;
         const bool diag = kt == nkt - 1;    // inside the diagonal key tile key 128 kt + col is visible iff col <= i - 128 kt
         const int lim = i - kt * kTile;
-        uint32_t s[kTile];               // the row's 128 scores (the softmax warps hold the registers for it)
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, s + ch * 32);
         tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&sm.s_free[grp]);      // the scores are in registers: S(ring + 2) may overwrite the buffer
         if (diag) {
 #pragma unroll
           for (int col = 0; col < kTile; ++col)
             if (col > lim) s[col] = 0xff800000u;   // -inf
         }
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        float mx[8];
 #pragma unroll
-        for (int col = 0; col < kTile; col += 8) {
-          mx0 = max3(mx0, __uint_as_float(s[col]), __uint_as_float(s[col + 1]));
-          mx1 = max3(mx1, __uint_as_float(s[col + 2]), __uint_as_float(s[col + 3]));
-          mx2 = max3(mx2, __uint_as_float(s[col + 4]), __uint_as_float(s[col + 5]));
-          mx3 = max3(mx3, __uint_as_float(s[col + 6]), __uint_as_float(s[col + 7]));
+        for (int c8 = 0; c8 < 8; ++c8) mx[c8] = max3(__uint_as_float(s[c8 * 2]), __uint_as_float(s[c8 * 2 + 1]), -INFINITY);
+#pragma unroll
+        for (int col = 16; col < kTile; col += 16) {
+#pragma unroll
+          for (int c8 = 0; c8 < 8; ++c8)
+            mx[c8] = max3(mx[c8], __uint_as_float(s[col + c8 * 2]), __uint_as_float(s[col + c8 * 2 + 1]));
         }
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc2;   // finite: column 0 of the tile is visible
-        // The maximum in use after the K tile before this one, from the thread that took it (the
-        // partner of this row, or this thread itself across a tile border). A tile's first K tile
-        // starts from -inf but still waits: the slot is one word per row.
-        float m_prev = -INFINITY;
-        if (ring > 0) ok = slot_wait(&sm.m_slot[row], (uint32_t)ring, &m_prev, abort_flag, a.status, code);
+        const float mxa = max3(mx[0], mx[1], mx[2]), mxb = max3(mx[3], mx[4], mx[5]);
+        const float mxs = max3(max3(mxa, mxb, mx[6]), mx[7], -INFINITY) * sc2;   // finite: column 0 of the tile is visible
+        // P(ring) goes to this group's P buffer, which PV(ring - 2) must have read. The wait comes
+        // before this thread publishes its maximum, so whoever reads that word knows that PV(ring - 2)
+        // is complete. That is what makes three things safe: the partner's parity wait for
+        // PV(ring - 1) in the rescale below (it reads the word of ring - 1, so PV(ring - 3), the phase
+        // before on that barrier, is complete); reusing a tile parity's word without a wait (a tile's
+        // first K tile R publishes after PV(R - 2), which needed the P of every K tile of the tile
+        // two back, written after their threads read the word); and reusing a row-sum slot four
+        // tiles on (PV(R - 2) is then past the first PV of the tile after the slot's, which waited
+        // for the epilogue to read it).
+        if (ok && ring >= 2) ok = mbar_wait(&sm.pv_done[grp], ph ^ 1, abort_flag, a.status, code);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        if (j == 0) m_prev = -INFINITY;
-        m_other = m_prev;
-        const bool need = mx > m_prev + kRescaleStep;      // always true on the first K tile of a tile
-        const float m_used = need ? mx : m_prev;
-        *reinterpret_cast<volatile unsigned long long*>(&sm.m_slot[row]) =
+        const bool need = mxs > m_prev + kRescaleStep;      // always true on the first K tile of a tile
+        const float m_used = need ? mxs : m_prev;
+        *reinterpret_cast<volatile unsigned long long*>(&sm.m_slot[tp][row]) =
             ((unsigned long long)(uint32_t)(ring + 1) << 32) | __float_as_uint(m_used);
         if (j > 0 && __any_sync(0xffffffffu, need)) {
-          // O may be rescaled once PV(ring - 1) is complete. (That barrier's phases are not followed
-          // one by one here, but it is exactly at this one: PV(ring - 4) had to be complete before
-          // S(ring - 1) was issued, and PV(ring + 2) comes after PV(ring), which needs the P this
-          // thread has yet to write.)
-          ok = mbar_wait(&sm.pv_done[(ring - 1) % kSBufs], ((ring - 1) / kSBufs) & 1, abort_flag, a.status, code);
+          // O may be rescaled once PV(ring - 1), the other group's, is complete: one phase behind at
+          // most (see above), and PV(ring + 1) cannot complete before this thread has written P(ring).
+          ok = mbar_wait(&sm.pv_done[grp ^ 1], ((ring - 1) >> 1) & 1, abort_flag, a.status, code);
           if (!ok) break;
           tc_fence_after();
           const float f = need ? ex2(m_prev - m_used) : 1.f;
@@ -385,7 +476,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         const float neg_m = -m_used;
         float part4[4] = {0.f, 0.f, 0.f, 0.f};
-        // P = exp2(S - m) as bf16 overwrites the first 64 columns of the buffer (S is in registers)
+        // P = exp2(S - m) as bf16
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint32_t p[16];
@@ -397,74 +488,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             part4[2 + (c2 & 1)] += p1;
             p[c2] = pack_bf16(p0, p1);
           }
-          tmem_st16(s_addr + ch * 16, p);
+          tmem_st16(p_addr + ch * 16, p);
         }
         l += (part4[0] + part4[1]) + (part4[2] + part4[3]);
-        // Group 0's row sum of the tile (relative to the maximum after K tile nkt - 2, which group 1
-        // reads for the last K tile) goes to the epilogue before the arrival for P(nkt - 2): the
-        // epilogue runs after PV(nkt - 1), which is issued after PV(nkt - 2), which follows that arrival.
-        if (grp == 0 && j == nkt - 2) sm.l_even[tp][row] = l;
+        // The group's row sum of the tile goes to the epilogue warps before the arrival for its last
+        // P of the tile: the tile's last PV, which the epilogue waits for, follows that arrival.
+        if (j == j_last)
+          *reinterpret_cast<volatile unsigned long long*>(&sm.fin[grp][it & (kFinSlots - 1)][row]) =
+              ((unsigned long long)__float_as_uint(l) << 32) | __float_as_uint(m_mine);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&sm.p_ready[sb]);
-      }
-      if (grp == 1) {
-        // Epilogue of the tile (group 1 took the last K tile, so m_mine is the final maximum). A
-        // thread whose wait ran out still goes to the barrier, and the barrier itself tells all
-        // 128 threads whether any of them did.
-        const int rl = ring0 + nkt - 1;
-        if (ok) ok = mbar_wait(&sm.pv_done[rl % kSBufs], (rl / kSBufs) & 1, abort_flag, a.status, code);
-        if (row == 0) bulk_wait_read_all();      // the stores of the tile before have read the staging tile
-        uint32_t any_bad;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 128, q;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(any_bad)
-            : "r"((uint32_t)(ok ? 0 : 1))
-            : "memory");
-        if (any_bad) { ok = false; break; }
-        tc_fence_after();
-        if (nkt >= 2) l += *reinterpret_cast<volatile float*>(&sm.l_even[tp][row]) * ex2(m_other - m_mine);
-        if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_mine + log2f(l)) * kLn2;
-        const float inv = 1.f / l;
-        // O leaves through shared memory and two TMA stores (rows past n are clipped by the store)
-        uint8_t* my_row = sm.o_stage + row * 128;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t o[64];
-          tmem_ld32(o_addr + hf * 64, o);
-          tmem_ld32(o_addr + hf * 64 + 32, o + 32);
-          tmem_wait_ld();
-          if (hf == 1) {           // the accumulator is in registers: the next tile may overwrite it
-            tc_fence_before();
-            mbar_arrive(&sm.o_free);
-          }
-#pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {     // 16-byte chunk ch of the row sits at ch ^ (row & 7): the 128-byte swizzle
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(o[ch * 8 + 0]) * inv, __uint_as_float(o[ch * 8 + 1]) * inv);
-            pk.y = pack_bf16(__uint_as_float(o[ch * 8 + 2]) * inv, __uint_as_float(o[ch * 8 + 3]) * inv);
-            pk.z = pack_bf16(__uint_as_float(o[ch * 8 + 4]) * inv, __uint_as_float(o[ch * 8 + 5]) * inv);
-            pk.w = pack_bf16(__uint_as_float(o[ch * 8 + 6]) * inv, __uint_as_float(o[ch * 8 + 7]) * inv);
-            *reinterpret_cast<uint4*>(my_row + hf * kHalfBytes + ((ch ^ (row & 7)) << 4)) = pk;
-          }
-        }
-        fence_proxy_async();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (row == 0) {
-          tma_store_4d(&map_o, sm.o_stage, 0, h, tl.r0, b);
-          tma_store_4d(&map_o, sm.o_stage + kHalfBytes, 64, h, tl.r0, b);
-          bulk_commit();
-        }
+        mbar_arrive(&sm.p_ready[grp]);
       }
       if (!ok) break;
       ring0 += nkt;
     }
-    if (grp == 1 && row == 0) bulk_wait_all();   // the last stores have left shared memory and are complete
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kSoftmaxWarps) {
+  if (warp == kWarpS) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -492,9 +534,8 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   cudaFuncAttributes fa;
   if ((e = cudaFuncGetAttributes(&fa, attn_tc_kernel)) != cudaSuccess) return e;
   if (fa.numRegs != kRegsLaunch) return cudaErrorInvalidConfiguration;
-  size_t smem = kSmemNeed + 1024;
-  if (smem > (size_t)smem_max) smem = (size_t)smem_max;
-  if (smem < kSmemNeed) return cudaErrorInvalidConfiguration;
+  const size_t smem = kSmemNeed + 1024;
+  if (smem > (size_t)smem_max) return cudaErrorInvalidConfiguration;
   e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   // One CTA per (sequence, head) when that fills the SMs evenly; otherwise deal each head's tiles

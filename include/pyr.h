@@ -63,7 +63,8 @@ typedef enum {
   PYR_ERR_ORDER = 6,            /* call out of the prefill/select/decode sequence  */
   PYR_ERR_CUDA = 7,             /* a CUDA runtime call failed                      */
   PYR_ERR_TIMEOUT = 8,          /* a bounded device-side wait ran out              */
-  PYR_ERR_SCRATCH_LIMIT = 9     /* problem exceeds the library's built-in scratch  */
+  PYR_ERR_SCRATCH_LIMIT = 9,    /* problem exceeds the library's built-in scratch  */
+  PYR_ERR_HOST_MEMORY = 10      /* the host-side handle could not be allocated     */
 } pyr_status_t;
 
 typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
@@ -223,22 +224,35 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, c
  * The split-K partial results go to an array compiled into the library
  * (4 MiB per GPU, resident on every GPU that loads the library until the
  * process exits). A call whose B * Hq * splits * (D + 2) floats exceed it
- * returns PYR_ERR_SCRATCH_LIMIT and launches nothing; the split count is
- * min(64, ceil(1184 / (B * Hkv)), ceil((len + 1) / 128)) before rounding the
- * rows per split up to 16, and with one split no scratch is used at all.
+ * returns PYR_ERR_SCRATCH_LIMIT and launches nothing. The split count is the
+ * one pyr_decode_attn uses: min(64, floor(2 * SMs / (B * Hkv)),
+ * ceil((len + 1) / 128)), at least 1, and then ceil((len + 1) / rows per
+ * split) with the rows per split rounded up to a multiple of 16; with one
+ * split no scratch is used at all.
  * All calls on a GPU share that array and it keeps the previous call's
  * contents (every slot is rewritten before it is read, so none needs
  * clearing): two calls whose kernels can overlap on the GPU - different
  * streams, or different threads - race on it; keep them on one stream or
- * order them with events. The first call on each GPU looks the array's device
- * address up, which is a CUDA runtime call outside the stream: make that
- * first call before any stream capture begins. No cudaMalloc, cudaFree or
- * other allocating routine is called, on any call.
+ * order them with events. The first call on each GPU, whatever its sizes,
+ * looks the array's device address up, which is a CUDA runtime call outside
+ * the stream: make that first call before any stream capture begins. No
+ * cudaMalloc, cudaFree or other allocating routine is called, on any call.
+ * A bounded device-side wait that runs out is recorded in a word beside the
+ * array; pyr_decode_attn_noalloc_status reads it. `out` of a call that hit one
+ * is undefined.
  */
 pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new, const void* v_new, void* out,
                                      void* k_cache, void* v_cache, int32_t batch, int32_t n_q_heads,
                                      int32_t n_kv_heads, int32_t head_dim, int32_t dtype, int32_t len,
                                      int32_t cap, float softmax_scale, void* stream);
+
+/*
+ * (No counterpart in the paper.) Synchronises `stream`, then reports whether any
+ * pyr_decode_attn_noalloc call on the current GPU recorded a device-side wait
+ * that ran out since the last report: *host_status is 0 or PYR_ERR_TIMEOUT, and
+ * the return value says the same. Reading clears the record. Allocates nothing.
+ */
+pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
 
 const char* pyr_status_string(pyr_status_t status);
 

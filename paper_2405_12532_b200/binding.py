@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libpyr.so")
 PYR_OK, PYR_ERR_INVALID, PYR_ERR_NULL, PYR_ERR_UNSUPPORTED, PYR_ERR_BUFFER_TOO_SMALL, \
     PYR_ERR_CAPACITY, PYR_ERR_ORDER, PYR_ERR_CUDA, PYR_ERR_TIMEOUT = range(9)
 PYR_ERR_SCRATCH_LIMIT = 9
+PYR_ERR_HOST_MEMORY = 10
 PYR_BF16, PYR_F32 = 0, 1
 PYR_FLAG_CUDA_CORE_PREFILL = 1
 
@@ -23,7 +24,7 @@ EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
     "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_status_string", "pyr_version", "pyr_launch_count",
-    "pyr_decode_attn_noalloc",
+    "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
 
 
@@ -78,6 +79,7 @@ def lib() -> C.CDLL:
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                               C.c_float, vp]
+        L.pyr_decode_attn_noalloc_status.argtypes = [vp, pi32]
         for name in EXPORTS:
             fn = getattr(L, name)
             if name not in ("pyr_status_string", "pyr_version", "pyr_launch_count"):
@@ -149,6 +151,14 @@ def decode_attn_noalloc(q, k_new, v_new, out, k_cache, v_cache, length: int, sof
     return lib().pyr_decode_attn_noalloc(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                          k_cache.data_ptr(), v_cache.data_ptr(), B, Hq, Hkv, D, dt, int(length),
                                          cap, float(softmax_scale), C.c_void_p(_stream_ptr(stream)))
+
+
+def decode_attn_noalloc_status(stream=None) -> int:
+    """pyr_decode_attn_noalloc_status: 0, or PYR_ERR_TIMEOUT if a wait of an earlier
+    no-alloc call ran out (synchronises the stream; reading clears the record)."""
+    w = C.c_int32(0)
+    lib().pyr_decode_attn_noalloc_status(C.c_void_p(_stream_ptr(stream)), C.byref(w))
+    return w.value
 
 
 def config_from_workload(w: dict, ratio, **over) -> dict:

@@ -22,6 +22,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 constexpr size_t kAlign = 256;
 
 std::atomic<uint64_t> g_launches{0};   // kernels launched by this process through the library
+std::atomic<int> g_sm_count[64];        // per device, 0 = not asked yet
 
 struct Layout {
   size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, total;
@@ -105,6 +106,23 @@ void plan(const pyr_config_t* c, Layout* lay) {
 
 }  // namespace
 
+namespace pyr {
+
+int device_sm_count() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int n = g_sm_count[dev].load();
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 0;
+    g_sm_count[dev].store(n);
+  }
+  return n;
+}
+
+void count_launches(int kernels) { g_launches += (uint64_t)kernels; }
+
+}  // namespace pyr
+
 struct pyr_cache {
   pyr_config_t cfg;
   std::vector<double> ratio;
@@ -160,6 +178,7 @@ const char* pyr_status_string(pyr_status_t s) {
     case PYR_ERR_CUDA: return "CUDA runtime error";
     case PYR_ERR_TIMEOUT: return "device-side wait timed out";
     case PYR_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library's built-in array holds";
+    case PYR_ERR_HOST_MEMORY: return "out of host memory";
   }
   return "unknown status";
 }
@@ -172,9 +191,13 @@ pyr_status_t pyr_cache_bytes(const pyr_config_t* cfg, size_t* bytes, size_t* ali
   pyr_status_t st = validate(cfg);
   if (st != PYR_OK) return st;
   if (!bytes) return PYR_ERR_NULL;
-  Layout lay;
-  plan(cfg, &lay);
-  *bytes = lay.total;
+  try {
+    Layout lay;
+    plan(cfg, &lay);
+    *bytes = lay.total;
+  } catch (...) {
+    return PYR_ERR_HOST_MEMORY;
+  }
   if (align) *align = kAlign;
   return PYR_OK;
 }
@@ -185,7 +208,8 @@ pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t byte
   if (!dev_buf || !out) return PYR_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(dev_buf) % kAlign) return PYR_ERR_INVALID;
   pyr_cache* c = new (std::nothrow) pyr_cache();
-  if (!c) return PYR_ERR_INVALID;
+  if (!c) return PYR_ERR_HOST_MEMORY;
+  try {
   c->cfg = *cfg;
   c->ratio.assign(cfg->ratio, cfg->ratio + cfg->n_layers);
   if (cfg->min_len) c->min_len.assign(cfg->min_len, cfg->min_len + cfg->n_layers);
@@ -204,6 +228,10 @@ pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t byte
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
   c->needs_init = true;
   c->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
+  } catch (...) {           // the host-side vectors could not be allocated
+    delete c;
+    return PYR_ERR_HOST_MEMORY;
+  }
   *out = c;
   return PYR_OK;
 }
@@ -402,7 +430,9 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   a.scale = c->scale; a.dtype = c->cfg.dtype;
   a.status = at<int>(c, c->lay.status);
   int splits = 1, rps = 0;
-  pyr::decode_split_rule(a.B, a.Hkv, a.len + 1, &splits, &rps);
+  const int sms = pyr::device_sm_count();
+  if (sms <= 0) return PYR_ERR_CUDA;
+  pyr::decode_split_rule(a.B, a.Hkv, a.len + 1, sms, &splits, &rps);
   a.splits = splits; a.rows_per_split = rps;
   if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
   g_launches += splits > 1 ? 2 : 1;

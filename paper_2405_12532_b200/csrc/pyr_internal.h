@@ -62,9 +62,9 @@ struct DecodeArgs {
 // `rows_per_split` (a multiple of 16) so that the grid is at most one wave of two CTAs per SM when
 // splitting is needed at all. The kernels are bandwidth-bound and every CTA pays about 5 us of
 // set-up and merging: a second, partial wave costs that again (measured: 13 us per launch).
-inline void decode_split_rule(int batch, int n_kv_heads, int total, int* splits_out, int* rows_per_split_out) {
+inline void decode_split_rule(int batch, int n_kv_heads, int total, int sms, int* splits_out, int* rows_per_split_out) {
   const long long pairs = (long long)batch * n_kv_heads;
-  int splits = (int)((148LL * 2) / pairs);
+  int splits = (int)(((long long)sms * 2) / pairs);
   const int max_by_rows = (total + 127) / 128;
   if (splits > max_by_rows) splits = max_by_rows;
   if (splits > kMaxDecodeSplits) splits = kMaxDecodeSplits;
@@ -74,6 +74,11 @@ inline void decode_split_rule(int batch, int n_kv_heads, int total, int* splits_
   *splits_out = (total + rps - 1) / rps;
   *rows_per_split_out = rps;
 }
+
+// Multiprocessors of the current device (asked once per device; 0 if the query fails).
+int device_sm_count();
+// Adds to the count that pyr_launch_count reports.
+void count_launches(int kernels);
 
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t s);
 cudaError_t launch_score_simt(const PrefillArgs& a, cudaStream_t s);

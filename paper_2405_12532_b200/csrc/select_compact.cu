@@ -244,7 +244,9 @@ cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s) {
   if (total == 0) return cudaSuccess;
   constexpr int U = 4;
   int64_t blocks = (total + 256 * U - 1) / (256 * U);
-  const int64_t cap = 148LL * 32;
+  const int sms = device_sm_count();
+  if (sms <= 0) return cudaErrorUnknown;
+  const int64_t cap = (int64_t)sms * 32;
   if (blocks > cap) blocks = cap;
   gather_kv_kernel<U><<<(unsigned)blocks, 256, 0, s>>>(a, lanes, total);
   return cudaGetLastError();

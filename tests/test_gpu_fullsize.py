@@ -17,11 +17,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 CASES = [
-    # workload, layers of its schedule to run, (sequence, group) samples per layer
-    ("7b_stack_8x2k", [1, 16, 31], 3),
-    ("7b_64x2k", [1, 31], 2),
-    ("13b_stack_32x4k", [1, 39], 2),
-    ("70b_gqa_16x8k", [1, 79], 2),
+    # workload, layers of its schedule to run (first, spread middle ones whose lengths are not
+    # multiples of 128, the short memory-bound ones at the end), (sequence, group) samples per layer
+    ("7b_stack_8x2k", [0, 1, 8, 16, 24, 28, 31], 6),
+    ("7b_64x2k", [0, 6, 12, 19, 26, 31], 6),
+    ("13b_stack_32x4k", [0, 7, 15, 23, 31, 39], 6),
+    ("70b_gqa_16x8k", [0, 16, 32, 48, 64, 79], 4),
 ]
 
 
@@ -122,3 +123,47 @@ def test_full_size_layer_against_oracle(name, layers, nsamp):
         del Q, K, V, out, cache
         torch.cuda.empty_cache()
     print(f"{name}: {exact} selections identical to the oracle's, {ties} differ only within the 1e-6 tie band")
+
+
+def test_chained_stack_all_layers_batch2():
+    """The 7B-shaped stack at batch 2 through all 32 layers of its schedule in ONE cache: the kept
+    set the GPU produced at layer l fixes what layer l + 1 receives (its length and its position
+    ids). Every call is compared with the oracle on the inputs the GPU call had (teacher forcing):
+    the kept set of sampled heads at every layer, the position chain of every group at every layer."""
+    w = dict(synth.CONFIGS["7b_stack_8x2k"], batch=2)
+    ratio = synth.ratio_schedule(w)
+    budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
+    B, H, D, L, N = w["batch"], w["n_q_heads"], w["head_dim"], w["recent_len"], w["prompt_len"]
+    cache = pb.PyrCache(device=DEV, **pb.config_from_workload(w, ratio))
+    pos_prev = np.broadcast_to(np.arange(N), (B, H, N)).copy()
+    wts = oracle.recent_weights(L)
+    exact = ties = 0
+    heads = [0, 5, 11, 17, 23, 31]
+    for l, bud in enumerate(budgets):
+        n, k, c = bud["n_in"], bud["k"], bud["c"]
+        assert cache.layer_info(l)["n_in"] == n
+        Q, K, V = synth.stack_layer_inputs(w, l, n, device=DEV)
+        out = torch.empty_like(Q)
+        cache.prefill_layer(l, Q, K, V, out)
+        n_out = cache.select_compact(l, K, V, out, D, out.stride(0), out.stride(1), D)
+        torch.cuda.synchronize()
+        assert n_out == bud["n_out"]
+        kept_all, pos_all = cache.kept(l)
+        kept_np, pos_np = kept_all.cpu().numpy(), pos_all.cpu().numpy()
+        for b in range(B):
+            for h in heads:
+                A, _ = oracle.attention_weights(synth.widen(Q[b, :, h]), synth.widen(K[b, :, h]),
+                                                oracle.softmax_scale_default(D), np.arange(c, n))
+                res = check_kept(kept_np[b, h], oracle.ensemble_score(A, L, wts), k, n, L)
+                exact += res == "exact"; ties += res == "tie"
+            # positions: every group, chained through the GPU's own kept sets
+            for h in range(H):
+                np.testing.assert_array_equal(pos_np[b, h], pos_prev[b, h][kept_np[b, h]])
+        pos_prev = np.stack([[pos_prev[b, h][kept_np[b, h]] for h in range(H)] for b in range(B)])
+        Kc, Vc = cache.kv(l)
+        idx = torch.from_numpy(kept_np[1, 7]).to(DEV).long()
+        assert torch.equal(Kc[1, 7, :n_out], K[1, idx, 7]) and torch.equal(Vc[1, 7, :n_out], V[1, idx, 7])
+    assert cache.status() == 0
+    cache.close()
+    print(f"chained 7b stack, batch 2, 32 layers: {exact} sampled selections identical to the oracle's, "
+          f"{ties} differ only within the 1e-6 tie band")

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2405_12532_b200 import binding as pb
 from paper_2405_12532_b200 import synth
 from parity_util import one_layer_cache, tol_for
@@ -46,13 +47,43 @@ def test_noalloc_decode_matches_handle_decode_twice(dtype, Hq, Hkv, D, B, n):
         torch.cuda.synchronize()
         err = (got.double() - want.double()).abs().max().item()
         assert err <= tol_for(dtype), err
+        # and against the CPU oracle on the same cache contents (rows 0..length+t-1 before the append)
+        for b in range(B):
+            ref, _, _ = oracle.decode_attention(synth.widen(q[b]), synth.widen(Kc[b, :, : length + t]),
+                                                synth.widen(Vc[b, :, : length + t]), synth.widen(kn[b]), synth.widen(vn[b]))
+            assert np.abs(synth.widen(got[b]) - ref).max() <= tol_for(dtype)
         assert torch.equal(Kmine[:, :, length + t], kn) and torch.equal(Vmine[:, :, length + t], vn)
         assert torch.equal(Kmine[:, :, : length + t + 1], Kc[:, :, : length + t + 1])
+    assert pb.decode_attn_noalloc_status() == 0
     cache.close()
 
 
+def test_noalloc_one_split_then_several():
+    """A short cache takes one split (no scratch), a longer one several: both against the oracle,
+    in that order, so the address lookup of the first call serves the second."""
+    Hq, Hkv, D, B = 4, 2, 128, 1
+    w = dict(n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, dtype="bf16", batch=B)
+    for length, cap in ((100, 128), (3000, 3072)):
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(length)
+        Kc = torch.randn(B, Hkv, cap, D, generator=gen, device=DEV).to(torch.bfloat16)
+        Vc = torch.randn(B, Hkv, cap, D, generator=gen, device=DEV).to(torch.bfloat16)
+        Kc[:, :, length:] = 0
+        Vc[:, :, length:] = 0
+        q, kn, vn = synth.decode_step_inputs(w, 0, length, device=DEV)
+        Kb, Vb = synth.widen(Kc[0, :, :length]), synth.widen(Vc[0, :, :length])
+        got = torch.full_like(q, float("nan"))
+        launches = pb.launch_count()
+        assert pb.decode_attn_noalloc(q, kn, vn, got, Kc, Vc, length) == pb.PYR_OK
+        torch.cuda.synchronize()
+        assert pb.launch_count() - launches == (1 if length < 128 else 2)
+        ref, _, _ = oracle.decode_attention(synth.widen(q[0]), Kb, Vb, synth.widen(kn[0]), synth.widen(vn[0]))
+        assert np.abs(synth.widen(got[0]) - ref).max() <= tol_for("bf16")
+    assert pb.decode_attn_noalloc_status() == 0
+
+
 def test_noalloc_rejects_what_does_not_fit():
-    B, Hq, Hkv, D, cap = 64, 64, 1, 128, 9000          # 64 * 64 * 64 splits * 130 floats > 4 MiB
+    B, Hq, Hkv, D, cap = 64, 64, 1, 128, 9000          # 64 * 64 * 4 splits * 130 floats > 4 MiB
     q = torch.zeros(B, Hq, D, device=DEV, dtype=torch.bfloat16)
     kn = torch.zeros(B, Hkv, D, device=DEV, dtype=torch.bfloat16)
     Kc = torch.zeros(B, Hkv, cap, D, device=DEV, dtype=torch.bfloat16)

@@ -17,6 +17,7 @@ from .pyramid import (  # noqa: F401
     gather_rows,
     prefill_layer,
     decode_attention,
+    generation_reselect,
     cache_capacities,
     cache_bytes,
     overlap_ratio,

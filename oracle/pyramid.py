@@ -11,8 +11,9 @@ textbook definition.
 Pins (tests/test_oracle_*.py): causal attention against a library routine,
 the ensemble score against explicit loops, a closed form and a row-sum
 invariant, the top-k against subset enumeration, budgets against the integer
-identities of the schedule, decode against one row of causal attention, cache
-bytes against the paper's Section 1 figure.
+identities of the schedule, decode against one row of causal attention, the
+generation-phase re-selection against the prefill step it must agree with and
+against explicit loops, cache bytes against the paper's Section 1 figure.
 
 parity unpinned: the absolute values of the ensemble score and the kept sets
 on real text. The paper prints no worked example of either.
@@ -255,6 +256,59 @@ def decode_attention(q, K_cache, V_cache, k_new, v_new, scale: float | None = No
         p = p / p.sum()
         out[h] = p @ Vc[g]
     return out, Kc, Vc
+
+
+def generation_reselect(Q_recent, K_cache, V_cache, k_keep: int, sel_groups: int,
+                        scale: float | None = None, w=None, pos=None):
+    """Generation-phase update of one sequence's PvC of one layer (Algorithm 1
+    with KV = cat([PvC_past, KV]); Section 4.1, Generation Phase: the recent
+    window slides over the generated tokens and the PvCs are re-selected "the
+    same as the prefill phase").
+
+    K_cache/V_cache [Hkv, len, D] hold the layer's cache in order: the context
+    rows, then the rows of the Lw most recent tokens. Q_recent [Lw, Hq, D]
+    holds those tokens' queries, oldest first. Reading taken: the attention
+    weights of the window queries are computed over the cache as it is now;
+    window query i sees the context and the window rows up to its own (row
+    c + i). The ensemble score, its pooling and the top-k are those of the
+    prefill step. Algorithm 1 selects only while len(KV) exceeds the layer's
+    bound: here, while the context is longer than k_keep.
+
+    Returns a dict: score [G, c], kept [G, n_out] (indices into the cache's
+    rows, ascending, the window last), K_kept/V_kept [Hkv, n_out, D],
+    pos_kept [G, n_out]; n_out = min(c, k_keep) + Lw.
+    """
+    Q_recent = np.asarray(Q_recent, dtype=F64)
+    K_cache = np.asarray(K_cache, dtype=F64)
+    V_cache = np.asarray(V_cache, dtype=F64)
+    Lw, Hq, D = Q_recent.shape
+    Hkv, n, _ = K_cache.shape
+    G = int(sel_groups)
+    assert G in (1, Hkv) and n >= Lw
+    c = n - Lw
+    r = Hq // Hkv
+    scale = softmax_scale_default(D) if scale is None else float(scale)
+    w = recent_weights(Lw) if w is None else np.asarray(w, dtype=F64)
+    pos = np.broadcast_to(np.arange(n, dtype=np.int64), (G, n)) if pos is None else np.asarray(pos)
+    k = min(c, int(k_keep))
+    E = np.zeros((Hq, c), dtype=F64)
+    window = np.arange(c, n)
+    for h in range(Hq):
+        q_rows = np.zeros((n, D), dtype=F64)
+        q_rows[c:] = Q_recent[:, h]                 # only the window's rows are read
+        A, _ = attention_weights(q_rows, K_cache[h // r], scale, window)
+        E[h] = ensemble_score(A, Lw, w)
+    score = pooled_scores(E, G) if c > 0 else np.zeros((G, 0), dtype=F64)
+    kept = np.stack([select_topk(score[g], k, n) for g in range(G)])
+    n_out = k + Lw
+    Kk = np.zeros((Hkv, n_out, D), dtype=F64)
+    Vk = np.zeros((Hkv, n_out, D), dtype=F64)
+    for g in range(Hkv):
+        idx = kept[g if G == Hkv else 0]
+        Kk[g] = gather_rows(K_cache[g], idx)
+        Vk[g] = gather_rows(V_cache[g], idx)
+    pk = np.stack([gather_rows(pos[g], kept[g]) for g in range(G)])
+    return {"score": score, "kept": kept, "K_kept": Kk, "V_kept": Vk, "pos_kept": pk}
 
 
 def cache_capacities(prompt_len, recent_len, ratio, max_new_tokens, min_len=None):

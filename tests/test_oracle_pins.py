@@ -322,6 +322,93 @@ def test_decode_equals_last_row_of_causal_attention():
     np.testing.assert_array_equal(Vc[:, n], V[n])
 
 
+# ---- generation-phase re-selection ----
+def _window_scores_by_loops(Qw, K, w, scale):
+    """Rectangular causal block by explicit loops: window query i (of Lw) sees cache rows 0..c+i."""
+    Lw, D = Qw.shape
+    n = K.shape[0]
+    c = n - Lw
+    E = np.zeros(c)
+    for i in range(Lw):
+        s = [scale * sum(Qw[i][d] * K[j][d] for d in range(D)) for j in range(c + i + 1)]
+        m = max(s)
+        e = [np.exp(x - m) for x in s]
+        z = sum(e)
+        for j in range(c):
+            E[j] += w[i] * e[j] / z
+    return E
+
+
+@pytest.mark.parametrize("G", [2, 1])
+def test_generation_reselect_by_loops_and_structure(G):
+    Hq, Hkv, D, n, Lw, k = 4, 2, 4, 17, 5, 6
+    Qw, K, V = _rand(Lw, Hq, D), _rand(Hkv, n, D), _rand(Hkv, n, D)
+    w = oracle.recent_weights(Lw)
+    out = oracle.generation_reselect(Qw, K, V, k, G, scale=0.8)
+    c = n - Lw
+    E = np.stack([_window_scores_by_loops(Qw[:, h], K[h // 2], w, 0.8) for h in range(Hq)])
+    per = Hq // G
+    for g in range(G):
+        np.testing.assert_allclose(out["score"][g], sum(E[g * per + i] for i in range(per)) / per, rtol=1e-12)
+        kept = out["kept"][g]
+        assert kept.shape == (k + Lw,) and np.all(np.diff(kept) > 0)
+        assert list(kept[k:]) == list(range(c, n))                      # the window is never evicted
+        dropped = np.setdiff1d(np.arange(c), kept)
+        assert out["score"][g][kept[:k]].min() >= out["score"][g][dropped].max()
+        np.testing.assert_array_equal(out["pos_kept"][g], kept)
+    for hk in range(Hkv):
+        idx = out["kept"][hk if G == Hkv else 0]
+        np.testing.assert_array_equal(out["K_kept"][hk], K[hk, idx])
+        np.testing.assert_array_equal(out["V_kept"][hk], V[hk, idx])
+
+
+def test_generation_reselect_is_the_prefill_operation():
+    # on an untouched prompt cache, with the last L prompt queries as the window, the generation-phase
+    # update must give the prefill step's scores and kept set (Section 4.1: "the same as the prefill phase")
+    B, n, Hq, Hkv, D, L, k = 1, 40, 4, 2, 8, 7, 11
+    Q, K, V = _rand(B, n, Hq, D), _rand(B, n, Hkv, D), _rand(B, n, Hkv, D)
+    pre = oracle.prefill_layer(Q, K, V, L, k, Hkv)
+    gen = oracle.generation_reselect(Q[0, n - L:], K[0].transpose(1, 0, 2), V[0].transpose(1, 0, 2), k, Hkv)
+    np.testing.assert_allclose(gen["score"], pre["score"][0], rtol=1e-12)
+    np.testing.assert_array_equal(gen["kept"], pre["kept"][0])
+    np.testing.assert_array_equal(gen["K_kept"], pre["K_kept"][0])
+
+
+def test_generation_reselect_edges_and_closed_form():
+    Hq, Hkv, D, n, Lw = 2, 2, 4, 30, 6
+    c = n - Lw
+    Qw, V = _rand(Lw, Hq, D), _rand(Hkv, n, D)
+    # a budget that covers the context evicts nothing
+    K = _rand(Hkv, n, D)
+    out = oracle.generation_reselect(Qw, K, V, c + 3, Hkv)
+    assert np.all(out["kept"] == np.arange(n))
+    np.testing.assert_array_equal(out["K_kept"], K)
+    # budget 0: only the window survives
+    out = oracle.generation_reselect(Qw, K, V, 0, 1)
+    assert list(out["kept"][0]) == list(range(c, n))
+    # identical keys: A[i, j] = 1 / (c + i + 1), so every context key scores sum_i w_i / (c + i + 1)
+    Kc = np.tile(_rand(1, 1, D), (Hkv, n, 1))
+    w = oracle.recent_weights(Lw)
+    out = oracle.generation_reselect(Qw, Kc, V, 4, Hkv)
+    want = sum(w[i] / (c + i + 1) for i in range(Lw))
+    np.testing.assert_allclose(out["score"], np.full((Hkv, c), want), rtol=1e-12)
+    assert list(out["kept"][0][:4]) == [0, 1, 2, 3]                     # ties go to the lower index
+
+
+def test_generation_reselect_then_decode_reads_the_gathered_cache():
+    Hq, Hkv, D, n, Lw, k = 4, 2, 8, 25, 5, 9
+    Qw, K, V = _rand(Lw, Hq, D), _rand(Hkv, n, D), _rand(Hkv, n, D)
+    out = oracle.generation_reselect(Qw, K, V, k, Hkv)
+    q, kn, vn = _rand(Hq, D), _rand(Hkv, D), _rand(Hkv, D)
+    got, Kc, _ = oracle.decode_attention(q, out["K_kept"], out["V_kept"], kn, vn)
+    assert Kc.shape[1] == k + Lw + 1
+    # head 0 by hand over its kept rows
+    idx = out["kept"][0]
+    s = np.concatenate([K[0, idx] @ q[0], [kn[0] @ q[0]]]) / np.sqrt(D)
+    p = np.exp(s - s.max()); p /= p.sum()
+    np.testing.assert_allclose(got[0], p @ np.concatenate([V[0, idx], vn[0][None]]), rtol=1e-12)
+
+
 # ---- cache bytes ----
 def test_cache_bytes_full_cache_closed_form_and_paper_figure():
     with open(os.path.join(GOLDEN, "kv_cache_7b_64x2k.txt")) as f:

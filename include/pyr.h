@@ -71,6 +71,8 @@ typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
 
 /* flags */
 #define PYR_FLAG_CUDA_CORE_PREFILL 1u /* bf16 prefill on the CUDA-core kernel (validation aid) */
+#define PYR_FLAG_GEN_RESELECT 2u      /* keep each layer's recent queries so that pyr_decode_reselect can
+                                         update the PvC during generation (Section 4.1, Generation Phase) */
 
 /*
  * Parameters of Algorithm 1 (recent window length L, minimum PvC lengths N_l,
@@ -203,6 +205,32 @@ pyr_status_t pyr_select_compact(pyr_cache_t* cache, int32_t layer, const void* k
  */
 pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, const void* k_new,
                              const void* v_new, void* out, void* stream);
+
+/*
+ * Section 4.1, Generation Phase, and Algorithm 1's branch for a cache that
+ * already holds past PvC: the recent window has slid over the generated tokens,
+ * and the layer's PvC is selected again "the same as the prefill phase". The
+ * attention weights of the window's queries (the last min(L, tokens so far)
+ * tokens; query i sees the context rows and the window rows up to its own) are
+ * taken over the layer's cache as it is now; their weighted average scores the
+ * context rows (all rows before the window), pooled per selection group; the
+ * layer's budget k_ctx of them is kept, ties to the lower row, and the cache's
+ * K and V rows are compacted in place, in order, the window last. The cache then
+ * holds k_ctx + window rows again: called every s decode steps it keeps a fixed
+ * number of PvCs per layer, so T only has to cover s steps.
+ * Nothing happens (and nothing is launched) while the context is not longer than
+ * k_ctx. *c_ctx (may be NULL) receives the number of context rows scored, *n_out
+ * (may be NULL) the rows the cache holds afterwards. pyr_cache_kept(layer) then
+ * gives the kept row indices [B, G, n_out] into the cache as it was (its position
+ * pointer repeats them: original positions are not tracked through generation)
+ * and pyr_cache_scores(layer) the pooled scores [B, G, c_ctx].
+ * Needs PYR_FLAG_GEN_RESELECT in the configuration (else PYR_ERR_UNSUPPORTED),
+ * which reserves a ring of L + max(T, 1) query rows per layer and makes
+ * pyr_prefill_layer (whose q rows must then be contiguous: strides Hq*D, D) and
+ * pyr_decode_attn record their queries. Allowed once every layer has been selected.
+ */
+pyr_status_t pyr_decode_reselect(pyr_cache_t* cache, int32_t layer, int32_t* c_ctx, int32_t* n_out,
+                                 void* stream);
 
 /*
  * Decode attention for callers that must not allocate device memory.

@@ -19,11 +19,12 @@ PYR_ERR_SCRATCH_LIMIT = 9
 PYR_ERR_HOST_MEMORY = 10
 PYR_BF16, PYR_F32 = 0, 1
 PYR_FLAG_CUDA_CORE_PREFILL = 1
+PYR_FLAG_GEN_RESELECT = 2
 
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_status_string", "pyr_version", "pyr_launch_count",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
 
@@ -77,6 +78,7 @@ def lib() -> C.CDLL:
         L.pyr_prefill_layer.argtypes = [vp, i32, vp, vp, vp, vp] + [i64] * 9 + [vp]
         L.pyr_select_compact.argtypes = [vp, i32, vp, vp, i64, i64, i64, vp, i64, i64, i64, i64, pi32, vp]
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+        L.pyr_decode_reselect.argtypes = [vp, i32, pi32, pi32, vp]
         L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                               C.c_float, vp]
         L.pyr_decode_attn_noalloc_status.argtypes = [vp, pi32]
@@ -268,6 +270,23 @@ class PyrCache:
             C.c_void_p(rows.data_ptr() if rows is not None else None), row_elems, rows_stride_b, rows_stride_n,
             rows_stride_g, C.byref(n_out), C.c_void_p(_stream_ptr(stream))), "pyr_select_compact")
         return n_out.value
+
+    def decode_reselect(self, layer: int, stream=None):
+        """pyr_decode_reselect: returns (context rows scored, rows the cache holds afterwards)."""
+        c_ctx, n_out = C.c_int32(0), C.c_int32(0)
+        _check(lib().pyr_decode_reselect(self.handle, layer, C.byref(c_ctx), C.byref(n_out),
+                                         C.c_void_p(_stream_ptr(stream))), "pyr_decode_reselect")
+        return c_ctx.value, n_out.value
+
+    def reselect_views(self, layer: int, c_ctx: int, n_out: int):
+        """(kept [B, G, n_out] int32, pooled scores [B, G, c_ctx] f32) of the last pyr_decode_reselect
+        of `layer` that selected."""
+        i, p = C.c_void_p(), C.c_void_p()
+        _check(lib().pyr_cache_kept(self.handle, layer, C.byref(i), C.byref(p)), "pyr_cache_kept")
+        sp = C.c_void_p()
+        _check(lib().pyr_cache_scores(self.handle, layer, C.byref(sp)), "pyr_cache_scores")
+        shape = (self.cfg.batch, self.cfg.sel_groups)
+        return self._view(i.value, shape + (n_out,), torch.int32), self._view(sp.value, shape + (c_ctx,), torch.float32)
 
     def decode_attn(self, layer: int, q, k_new, v_new, out, stream=None):
         assert q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous() and out.is_contiguous()

@@ -15,6 +15,7 @@ namespace {
 struct LayerPlan {
   int n_in, c, k, n_out, cap;
   size_t k_off, v_off;   // byte offsets into the device buffer
+  size_t q_off;          // ring of recent queries (generation-phase re-selection only)
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -25,7 +26,8 @@ std::atomic<uint64_t> g_launches{0};   // kernels launched by this process throu
 std::atomic<int> g_sm_count[64];        // per device, 0 = not asked yet
 
 struct Layout {
-  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, total;
+  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, gen_part, total;
+  int q_ring;            // rows of a layer's query ring (0: no generation-phase re-selection)
   std::vector<LayerPlan> layers;
 };
 
@@ -68,7 +70,10 @@ void plan(const pyr_config_t* c, Layout* lay) {
   size_t off = 0;
   lay->status = off; off = align_up(off + pyr::kStatusWords * sizeof(int), kAlign);
   lay->w = off;      off = align_up(off + (size_t)L * 4, kAlign);
-  lay->score = off;  off = align_up(off + B * G * (size_t)(c0 > 0 ? c0 : 1) * 4, kAlign);
+  const bool gen = (c->flags & PYR_FLAG_GEN_RESELECT) != 0;
+  // generation-phase re-selection scores up to c_0 + T context rows (the kept context plus the decode rows)
+  const size_t c_max = (size_t)(c0 > 0 ? c0 : 1) + (gen ? (size_t)c->max_new_tokens : 0);
+  lay->score = off;  off = align_up(off + B * G * c_max * 4, kAlign);
   // per-head partial scores of the tensor-core score kernel (bf16, head_dim 128 only)
   lay->score_part = off;
   if (c->dtype == PYR_BF16 && D == 128 && c0 > 0)
@@ -81,6 +86,9 @@ void plan(const pyr_config_t* c, Layout* lay) {
   if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * D * 4, kAlign);
   lay->part_ml = off;
   if (c->max_new_tokens > 0) off = align_up(off + B * Hq * pyr::kMaxDecodeSplits * 2 * 4, kAlign);
+  lay->gen_part = off;
+  if (gen) off = align_up(off + B * Hq * (size_t)pyr::gen_score_qtiles(L) * c_max * 4, kAlign);
+  lay->q_ring = gen ? L + (c->max_new_tokens > 0 ? c->max_new_tokens : 1) : 0;
   lay->layers.resize(c->n_layers);
   int n_in = N;
   for (int l = 0; l < c->n_layers; ++l) {
@@ -99,6 +107,8 @@ void plan(const pyr_config_t* c, Layout* lay) {
     const size_t bytes = B * Hkv * (size_t)p.cap * D * eb;
     p.k_off = off; off = align_up(off + bytes, kAlign);
     p.v_off = off; off = align_up(off + bytes, kAlign);
+    p.q_off = off;
+    if (gen) off = align_up(off + B * (size_t)lay->q_ring * Hq * D * eb, kAlign);
     n_in = p.n_out;
   }
   lay->total = off;
@@ -131,6 +141,7 @@ struct pyr_cache {
   Layout lay;
   char* base;
   std::vector<int> len_now;
+  std::vector<long long> q_count;   // queries written to each layer's ring so far
   int next_layer;     // layer whose prefill (phase 0) or select (phase 1) comes next
   int phase;
   int pos_cur;        // which of pos0/pos1 holds the positions of the last selection
@@ -225,6 +236,7 @@ pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t byte
   if (bytes < c->lay.total) { delete c; return PYR_ERR_BUFFER_TOO_SMALL; }
   c->base = static_cast<char*>(dev_buf);
   c->len_now.assign(cfg->n_layers, 0);
+  c->q_count.assign(cfg->n_layers, 0);
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
   c->needs_init = true;
   c->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
@@ -246,6 +258,7 @@ pyr_status_t pyr_cache_reset(pyr_cache_t* c, void* stream) {
   if (!c) return PYR_ERR_NULL;
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
   std::fill(c->len_now.begin(), c->len_now.end(), 0);
+  std::fill(c->q_count.begin(), c->q_count.end(), 0);
   return device_init(c, static_cast<cudaStream_t>(stream));
 }
 
@@ -347,6 +360,19 @@ pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, con
     if (e != cudaSuccess) return PYR_ERR_CUDA;
     g_launches += tc_score ? 2 : 1;
   }
+  if (c->lay.q_ring > 0) {
+    // the window's queries go to the layer's ring: the generation phase re-scores the cache with them
+    const int eb = c->cfg.dtype == PYR_BF16 ? 2 : 4;
+    const int Lw = p.n_in - p.c;
+    const int64_t row_bytes = (int64_t)c->cfg.n_q_heads * D * eb;
+    if (qsh != D || qsn != (int64_t)c->cfg.n_q_heads * D) return PYR_ERR_UNSUPPORTED;   // rows must be contiguous
+    e = pyr::launch_copy_rows(static_cast<const char*>(q) + (int64_t)p.c * qsn * eb, c->base + p.q_off, qsb * eb,
+                              qsn * eb, (int64_t)c->lay.q_ring * row_bytes, row_bytes, c->cfg.batch, Lw,
+                              (int)row_bytes, s);
+    if (e != cudaSuccess) return PYR_ERR_CUDA;
+    g_launches += 1;
+    c->q_count[layer] = Lw;
+  }
   c->phase = 1;
   c->last_prefilled = layer;
   return PYR_OK;
@@ -398,6 +424,7 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
     ra.rows = rows; ra.idx = sa.idx; ra.stride_b = rsb; ra.stride_n = rsn; ra.stride_g = rsg;
     ra.row_elems = row_elems; ra.B = c->cfg.batch; ra.G = c->cfg.sel_groups; ra.n_out = p.n_out;
     ra.elem_bytes = eb;
+    ra.idx_div = 1;
     if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
     g_launches += 1;
   }
@@ -437,6 +464,71 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   if (pyr::launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PYR_ERR_CUDA;
   g_launches += splits > 1 ? 2 : 1;
   c->len_now[layer] += 1;
+  if (c->lay.q_ring > 0) {
+    const int eb = c->cfg.dtype == PYR_BF16 ? 2 : 4;
+    const int64_t row_bytes = (int64_t)c->cfg.n_q_heads * c->cfg.head_dim * eb;
+    const int slot = (int)(c->q_count[layer] % c->lay.q_ring);
+    if (pyr::launch_copy_rows(q, c->base + p.q_off + (int64_t)slot * row_bytes, row_bytes, row_bytes,
+                              (int64_t)c->lay.q_ring * row_bytes, row_bytes, c->cfg.batch, 1, (int)row_bytes,
+                              static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      return PYR_ERR_CUDA;
+    g_launches += 1;
+    c->q_count[layer] += 1;
+  }
+  return PYR_OK;
+}
+
+pyr_status_t pyr_decode_reselect(pyr_cache_t* c, int32_t layer, int32_t* c_ctx, int32_t* n_out, void* stream) {
+  if (!c) return PYR_ERR_NULL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return PYR_ERR_INVALID;
+  if (c->lay.q_ring == 0) return PYR_ERR_UNSUPPORTED;
+  if (c->next_layer != c->cfg.n_layers) return PYR_ERR_ORDER;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const LayerPlan& p = c->lay.layers[layer];
+  const int L = c->cfg.recent_len;
+  const int len = c->len_now[layer];
+  const long long qn = c->q_count[layer];
+  const int Lw = (int)(qn < L ? qn : L);
+  const int ctx = len - Lw;
+  if (c_ctx) *c_ctx = ctx;
+  if (ctx <= p.k) {                       // Algorithm 1 selects only while the cache exceeds its bound
+    if (n_out) *n_out = len;
+    return PYR_OK;
+  }
+  const int eb = c->cfg.dtype == PYR_BF16 ? 2 : 4;
+  const int D = c->cfg.head_dim;
+  pyr::GenScoreArgs ga;
+  ga.qwin = c->base + p.q_off; ga.kc = c->base + p.k_off;
+  ga.part = at<float>(c, c->lay.gen_part); ga.score = at<float>(c, c->lay.score);
+  ga.w = at<float>(c, c->lay.w) + (L - Lw);
+  ga.B = c->cfg.batch; ga.Hq = c->cfg.n_q_heads; ga.Hkv = c->cfg.n_kv_heads; ga.D = D; ga.G = c->cfg.sel_groups;
+  ga.R = c->lay.q_ring; ga.start = (int)((qn - Lw) % c->lay.q_ring); ga.Lw = Lw; ga.len = len; ga.cap = p.cap; ga.c = ctx;
+  ga.scale = c->scale; ga.dtype = c->cfg.dtype;
+  if (pyr::launch_gen_score(ga, s) != cudaSuccess) return PYR_ERR_CUDA;
+
+  pyr::SelectArgs sa;
+  sa.score = ga.score;
+  sa.idx = at<int32_t>(c, c->lay.idx);
+  sa.pos_in = nullptr;                    // positions are not tracked through the generation phase
+  sa.pos_out = at<int32_t>(c, c->pos_cur ? c->lay.pos0 : c->lay.pos1);
+  sa.B = c->cfg.batch; sa.G = c->cfg.sel_groups; sa.n = len; sa.c = ctx; sa.k = p.k;
+  if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
+  c->pos_cur ^= 1;
+  c->last_selected = layer;
+  c->last_prefilled = layer;             // the score buffer now holds this layer's generation-phase scores
+
+  // K and V rows move up in place: kept indices ascend, so a row's destination lies at or below its source
+  pyr::RowsArgs ra;
+  ra.idx = sa.idx; ra.stride_b = (int64_t)c->cfg.n_kv_heads * p.cap * D; ra.stride_n = D;
+  ra.stride_g = (int64_t)p.cap * D; ra.row_elems = D; ra.B = c->cfg.batch; ra.G = c->cfg.n_kv_heads;
+  ra.n_out = p.k + Lw; ra.elem_bytes = eb; ra.idx_div = c->cfg.n_kv_heads / c->cfg.sel_groups;
+  ra.rows = c->base + p.k_off;
+  if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
+  ra.rows = c->base + p.v_off;
+  if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
+  g_launches += 5;
+  c->len_now[layer] = p.k + Lw;
+  if (n_out) *n_out = p.k + Lw;
   return PYR_OK;
 }
 

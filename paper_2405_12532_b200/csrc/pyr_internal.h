@@ -45,6 +45,19 @@ struct RowsArgs {
   int64_t stride_b, stride_n, stride_g;   // elements
   int64_t row_elems;
   int B, G, n_out, elem_bytes;
+  int idx_div;         // consecutive row groups that share one index list (1: a list per group)
+};
+
+// Generation-phase score of a layer's cache from its window of recent queries.
+struct GenScoreArgs {
+  const void* qwin;    // [B, R, Hq, D]: ring of the most recent queries; window query i is slot (start + i) % R
+  const void* kc;      // [B, Hkv, cap, D]
+  float* part;         // [B, Hq, query tiles, c] per-head partial scores
+  float* score;        // [B, G, c] pooled
+  const float* w;      // [Lw] device, oldest first
+  int B, Hq, Hkv, D, G, R, start, Lw, len, cap, c;   // c = len - Lw context rows
+  float scale;
+  int dtype;
 };
 
 struct DecodeArgs {
@@ -93,5 +106,10 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s);
 cudaError_t launch_compact_rows(const RowsArgs& a, cudaStream_t s);
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s);
+int gen_score_qtiles(int Lw);
+cudaError_t launch_gen_score(const GenScoreArgs& a, cudaStream_t s);     // two kernels
+// rows of row_bytes (a multiple of 16) per batch entry, byte strides
+cudaError_t launch_copy_rows(const void* src, void* dst, int64_t src_sb, int64_t src_sn, int64_t dst_sb,
+                             int64_t dst_sn, int B, int rows, int row_bytes, cudaStream_t s);
 
 }  // namespace pyr

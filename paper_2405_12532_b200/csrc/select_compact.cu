@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, i
   if (lanes <= 0) return;
   char* base = static_cast<char*>(a.rows) + ((int64_t)b * a.stride_b + (int64_t)g * a.stride_g) * eb + (int64_t)lane0 * 16;
   const int64_t row_bytes = a.stride_n * eb;
-  const int32_t* idx = a.idx + (int64_t)bg * a.n_out;
+  const int32_t* idx = a.idx + ((int64_t)b * (a.G / a.idx_div) + g / a.idx_div) * a.n_out;
   const int rows_per_iter = (kRowThreads * kRowUnroll) / lanes;   // lanes <= kRowThreads
   const int t = threadIdx.x;
   // Chunk i + 1 is read while chunk i is written: the sources of a later chunk lie above every

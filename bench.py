@@ -31,10 +31,32 @@ from paper_2405_12532_b200 import dist as pdist
 from paper_2405_12532_b200 import synth
 
 METRIC = "prefill tokens/s + decode tokens/s at 7B shapes 64x2k"
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch divided by its algorithmic bytes
-# (542.04 MB / 537.13 MB in profiles/decode_kernel_7b_2k_batch16.txt). Set to None when the kernel changes.
-DECODE_TRAFFIC_RATIO = 542.04 / 537.13
+UNIT = "tokens/s (prefill of the attention path, all layers incl. select+compact; no linear layers, no weight reads)"
+SCOPE = ("attention path only: per-layer Q/K/V are inputs; a full model's projections, MLP and weight reads "
+         "are not in the step")
 DEFAULT_WORKLOAD = "7b_64x2k"
+PROFILES = os.path.join(ROOT, "profiles")
+
+
+def traffic_ratio(summary: str):
+    """DRAM bytes per algorithmic byte of a kernel, from the ncu summary under profiles/ that
+    states it (`traffic_ratio: R`) together with the hash of the source file the kernel was
+    built from (`source_sha1: FILE HASH`). None when there is no such line or the source has
+    changed since the capture."""
+    import hashlib
+    import re
+    path = os.path.join(PROFILES, summary)
+    if not os.path.exists(path):
+        return None
+    text = open(path).read()
+    m = re.search(r"^traffic_ratio:\s*([0-9.]+)", text, re.M)
+    h = re.search(r"^source_sha1:\s*(\S+)\s+([0-9a-f]{40})", text, re.M)
+    if not m or not h:
+        return None
+    src = os.path.join(ROOT, "paper_2405_12532_b200", "csrc", h.group(1))
+    if not os.path.exists(src) or hashlib.sha1(open(src, "rb").read()).hexdigest() != h.group(2):
+        return None
+    return float(m.group(1))
 
 
 def measured_peaks():
@@ -102,7 +124,8 @@ class ClockSampler:
 class Workload:
     """Device-resident synthetic inputs and the call sequence of one step."""
 
-    def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1, batch: int = 0):
+    def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1, batch: int = 0,
+                 reselect_every: int = 0):
         from paper_2405_12532_b200 import binding as pb
         self.pb = pb
         self.name = name
@@ -116,7 +139,9 @@ class Workload:
             w["max_new_tokens"] = decode_steps
         if batch > 0:             # profiling aid: a smaller batch keeps an ncu capture small
             w["batch"] = batch
-        self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio))
+        self.reselect_every = reselect_every      # generation-phase PvC update every so many decode steps (0: never)
+        flags = pb.PYR_FLAG_GEN_RESELECT if reselect_every else 0
+        self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio, flags=flags))
         self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
         B, N, Hq, Hkv, D = w["batch"], w["prompt_len"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
         self.dt = synth.torch_dtype(w["dtype"])
@@ -168,11 +193,32 @@ class Workload:
             q, kn, vn = self.dec_in[t % len(self.dec_in)]
             for l in range(self.w["n_layers"]):
                 c.decode_attn(l, q, kn, vn, self.dec_out)
+            if self.reselect_every and (t + 1) % self.reselect_every == 0:
+                for l in range(self.w["n_layers"]):
+                    c.decode_reselect(l)
 
     # ---- algorithmic work, from the schedule
     def prefill_flops(self):
         w = self.w
         return sum(w["batch"] * w["n_q_heads"] * 2 * w["head_dim"] * L["n_in"] * (L["n_in"] + 1) for L in self.layers)
+
+    def prefill_roofline_seconds(self, tflops: float, hbm_gbs: float):
+        """Sum over layers of max(flops / tensor peak, compulsory Q+K+V+O bytes / HBM bandwidth):
+        the short layers deep in the pyramid are bound by their traffic, not by the contraction."""
+        w = self.w
+        B, Hq, Hkv, D = w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
+        t = 0.0
+        for L in self.layers:
+            n = L["n_in"]
+            flops = B * Hq * 2 * D * n * (n + 1)
+            byts = B * n * (2 * Hq + 2 * Hkv) * D * self.eb
+            t += max(flops / (tflops * 1e12), byts / (hbm_gbs * 1e9))
+        return t
+
+    def prefill_bytes(self):
+        w = self.w
+        return sum(w["batch"] * L["n_in"] * (2 * w["n_q_heads"] + 2 * w["n_kv_heads"]) * w["head_dim"] * self.eb
+                   for L in self.layers)
 
     def select_compact_bytes(self):
         w = self.w
@@ -196,15 +242,18 @@ class Workload:
         for L in self.layers:
             n_out = L["k_ctx"] + min(w["recent_len"], L["n_in"])
             for t in range(self.T):
-                tot += 2 * w["batch"] * w["n_kv_heads"] * (n_out + t + 1) * w["head_dim"] * self.eb
+                grown = t % self.reselect_every if self.reselect_every else t   # rows appended since the last update
+                tot += 2 * w["batch"] * w["n_kv_heads"] * (n_out + grown + 1) * w["head_dim"] * self.eb
         return tot
 
 
-def run_ours(args, rank, world, local_rank):
+def run_ours(args, rank, world, local_rank, workload=None):
     from paper_2405_12532_b200 import binding as pb
+    name = workload or args.workload
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
-    wl = Workload(args.workload, device, layers=args.layers, decode_steps=args.decode_steps, batch=args.batch)
+    wl = Workload(name, device, layers=args.layers, decode_steps=args.decode_steps, batch=args.batch,
+                  reselect_every=args.reselect_every)
     w = wl.w
     nL = w["n_layers"]
     hbm, tf_burst, tf_sust, peak_src = measured_peaks()
@@ -256,47 +305,62 @@ def run_ours(args, rank, world, local_rank):
     roof_dec = None
     if T > 0:
         ach = K * dec_bytes / t_dec / 1e9
+        rr = traffic_ratio("decode_kernel_7b_2k_batch16.txt")
         roof_dec = {"kernel": "decode_kernel", "bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s",
-                    "frac": ach / hbm, "traffic": DECODE_TRAFFIC_RATIO * dec_bytes / dec_launches,
+                    "frac": ach / hbm, "traffic": rr * dec_bytes / dec_launches if rr else None,
                     "traffic_note": "dram read+write bytes per launch, scaled from one ncu capture at batch 16 "
                                     "(profiles/decode_kernel_7b_2k_batch16.txt) by the rows streamed",
                     "peak_source": f"of {peak_src}",
                     "launches": K * dec_launches, "avg_launch_us": t_dec / (K * dec_launches) * 1e6,
-                    "algorithmic_bytes_per_launch": dec_bytes / dec_launches}
+                    "algorithmic_bytes_per_launch": dec_bytes / dec_launches,
+                    "reselect_every": args.reselect_every or None}
     ach_tf = K * wl.prefill_flops() / t_attn / 1e12
+    t_roof = wl.prefill_roofline_seconds(tf_burst, hbm)
+    t_roof_s = wl.prefill_roofline_seconds(tf_sust, hbm)
+    rr = traffic_ratio("attn_tc_kernel_7b_2k_batch16.txt")
     roof_pre = {"kernel": "prefill attention + score", "bound": "tensor", "achieved": ach_tf, "peak": tf_burst,
                 "unit": "TFLOP/s", "frac": ach_tf / tf_burst, "frac_of_sustained": ach_tf / tf_sust,
-                "traffic": None, "peak_source": f"of {peak_src}", "launches": K * nL * 2,
-                "avg_layer_us": t_attn / (K * nL) * 1e6}
+                # per layer max(flops / tensor peak, Q+K+V+O bytes / HBM bandwidth), summed, over the measured time
+                "frac_of_layer_roofline": K * t_roof / t_attn, "frac_of_layer_roofline_sustained": K * t_roof_s / t_attn,
+                "traffic": rr * wl.prefill_bytes() / nL if rr else None,
+                "traffic_note": "dram bytes of the attention kernel per launch (average layer), scaled from one ncu "
+                                "capture at batch 16 by the Q+K+V+O bytes",
+                "peak_source": f"of {peak_src}", "launches": K * nL * 2, "avg_layer_us": t_attn / (K * nL) * 1e6}
     ach_sel = K * wl.select_compact_bytes() / t_sel / 1e9
+    rr = traffic_ratio("gather_kv_kernel_7b_2k_batch16.txt")
     roof_sel = {"kernel": "select + gather + compact", "bound": "hbm", "achieved": ach_sel, "peak": hbm,
-                "unit": "GB/s", "frac": ach_sel / hbm, "traffic": None, "peak_source": f"of {peak_src}",
-                "avg_layer_us": t_sel / (K * nL) * 1e6}
+                "unit": "GB/s", "frac": ach_sel / hbm,
+                "traffic": rr * wl.select_compact_bytes() / nL if rr else None,
+                "traffic_note": "dram bytes per layer, scaled from the gather kernel's ncu capture at batch 16",
+                "peak_source": f"of {peak_src}", "avg_layer_us": t_sel / (K * nL) * 1e6}
     dominant = roof_dec if (roof_dec and t_dec >= t_attn) else roof_pre
     line = {
-        "metric": METRIC, "value": prefill_tps, "unit": "tokens/s (prefill, all layers incl. select+compact)",
+        "metric": METRIC, "value": prefill_tps, "unit": UNIT,
         "decode_tokens_per_s": decode_tps,
         "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": t_all / K * 1e3,
         "ms_prefill": t_pre / K * 1e3, "ms_decode": t_dec / K * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w["dtype"], "data": "synthetic",
-        "config": {"workload": args.workload, "layers": nL, "batch_per_gpu": B, "prompt_len": N,
+        "config": {"workload": name, "scope": SCOPE, "layers": nL, "batch_per_gpu": B, "prompt_len": N,
                    "recent_len": w["recent_len"], "decode_steps": T, "sel_groups": w["sel_groups"],
                    "heads": w["n_q_heads"], "kv_heads": w["n_kv_heads"], "head_dim": w["head_dim"],
                    "ratio": "geometric 1.0->%.2f" % wl.ratio[-1],
+                   "reselect_every": args.reselect_every or None,
                    "l2": "inputs larger than L2 (each of Q, K, V and the cache is >= 1 GB)"},
         "roofline": dominant, "roofline_prefill": roof_pre, "roofline_select_compact": roof_sel,
         "roofline_decode": roof_dec,
         "gpu_launches": launches, "wall_s": wall, "clocks": clocks, "e2e": e2e,
-        "cpu_baseline": cpu_baseline(args.workload) if not args.no_cpu else None,
+        "cpu_baseline": cpu_baseline(name) if not args.no_cpu else None,
     }
-    print(json.dumps(line))
+    print(json.dumps(line), flush=True)
+    wl.cache.close()
 
 
 def run_e2e(wl, args, barrier, world):
     """The same step driven from pinned host buffers: each layer's Q/K/V are
     copied host->device before its calls, the last layer's attention output and
-    every decode output are copied back."""
+    every decode output are copied back. `value` is the headline metric (prefill
+    tokens/s) with those copies inside the timed region."""
     w = wl.w
     steps = max(1, min(args.steps, args.e2e_steps))
     host_pool = [tuple(x.to("cpu").pin_memory() for x in qkv) for qkv in wl.pool[:1]]
@@ -308,10 +372,13 @@ def run_e2e(wl, args, barrier, world):
     c = wl.cache
     nL = w["n_layers"]
     h2d = d2h = 0
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
 
-    def step(count):
+    def step(count, mk=None):
         nonlocal h2d, d2h
         c.reset()
+        if mk:
+            mk[0].record()
         for l in range(nL):
             n = wl.layers[l]["n_in"]
             for src, dst in ((hq, dq), (hk, dk), (hv, dv)):
@@ -329,6 +396,8 @@ def run_e2e(wl, args, barrier, world):
             out_host[bi, :n_last].copy_(wl.out[bi, :n_last], non_blocking=True)
         if count:
             d2h += wl.out[:, :n_last].numel() * wl.out.element_size()
+        if mk:
+            mk[1].record()
         q, kn, vn = wl.dec_in[0]
         hq1, hk1, hv1 = dec_host[0]
         for t in range(wl.T):
@@ -339,19 +408,24 @@ def run_e2e(wl, args, barrier, world):
                 if count:
                     h2d += (q.numel() + kn.numel() + vn.numel()) * q.element_size()
                     d2h += wl.dec_out.numel() * wl.dec_out.element_size()
+            if wl.reselect_every and (t + 1) % wl.reselect_every == 0:
+                for l in range(nL):
+                    c.decode_reselect(l)
+        if mk:
+            mk[2].record()
 
     step(False)
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        step(True)
-    e1.record()
+    for i in range(steps):
+        step(True, marks[i])
     barrier()
-    t = pdist.max_over_ranks([e0.elapsed_time(e1) / 1e3], world, wl.device)[0]
+    t_pre = sum(m[0].elapsed_time(m[1]) for m in marks) / 1e3
+    t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
+    t_pre, t_dec = pdist.max_over_ranks([t_pre, t_dec], world, wl.device)
     B, N, T = w["batch"], w["prompt_len"], w["max_new_tokens"]
-    return {"value": world * steps * B * (N + T) / t, "unit": "tokens/s (prompt + generated, whole step from host buffers)",
-            "steps": steps, "ms_per_step": t / steps * 1e3,
+    return {"value": world * steps * B * N / t_pre, "unit": UNIT,
+            "decode_tokens_per_s": world * steps * B * T / t_dec if T > 0 and t_dec > 0 else None,
+            "steps": steps, "ms_per_step": (t_pre + t_dec) / steps * 1e3, "ms_prefill": t_pre / steps * 1e3,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps}
 
 
@@ -394,8 +468,8 @@ def oracle_sample(workload: str, layers=None):
 
 def cpu_baseline(workload: str):
     t, desc, tps, cores = oracle_sample(workload)
-    return {"value": tps, "unit": "tokens/s (prefill, estimated from the sample)", "cores": cores, "kind": "oracle",
-            "sample": desc, "sample_seconds": t}
+    return {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "sample_seconds": t,
+            "note": "estimated from the sample"}
 
 
 def run_reference(args, rank, world):
@@ -413,14 +487,59 @@ def run_reference(args, rank, world):
             per_step.append((time.perf_counter() - t0, tps))
     value = statistics.mean(x[1] for x in per_step)
     ms = statistics.mean(x[0] for x in per_step) * 1e3
-    unit = "tokens/s (prefill, estimated from the sample)"
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": world,
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload},
-            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": desc},
-            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
-    print(json.dumps(line))
+            "config": {"workload": args.workload, "scope": SCOPE},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                             "note": "estimated from the sample"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_dry(args, rank, world):
+    """Launch-path check without a GPU: the ranks meet on gloo, agree on the slowest rank's time
+    as the timed run does, and rank 0 prints what the launch looked like."""
+    pdist.init("gloo") if world > 1 else None
+    pdist.barrier(world)
+    mx = pdist.max_over_ranks([1.0 + rank], world)
+    lo, hi = synth.shard_batch(synth.CONFIGS[args.workload]["batch"] * world, world, rank)
+    pdist.barrier(world)
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "slowest_rank_seconds": mx[0],
+                          "rank0_sequences": [lo, hi], "workload": args.workload}), flush=True)
+
+
+def run(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.dry_run:
+        try:
+            run_dry(args, rank, world)
+        finally:
+            if world > 1 and torch.distributed.is_initialized():
+                torch.distributed.destroy_process_group()
+        return
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        pdist.init("nccl", torch.device("cuda", local_rank))
+    try:
+        names = list(synth.CONFIGS) if args.workload == "all" else [args.workload]
+        for name in names:          # "all": one line per workload, back to back
+            run_ours(args, rank, world, local_rank, name)
+            torch.cuda.empty_cache()
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+def _spawned(rank, args, port):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(args.gpus), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    run(args)
 
 
 def main():
@@ -429,27 +548,27 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(synth.CONFIGS))
-    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(synth.CONFIGS) + ["all"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--reselect-every", type=int, default=0,
+                    help="generation-phase PvC update of every layer every so many decode steps (0: never)")
+    ap.add_argument("--dry-run", action="store_true", help="launch path only (gloo, no GPU work)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: only the first LAYERS layers")
     ap.add_argument("--decode-steps", type=int, default=-1, help="profiling aid: override the decode steps")
     ap.add_argument("--batch", type=int, default=0, help="profiling aid: override the batch size")
     args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
-        run_reference(args, rank, world)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        # not under a launcher: start one rank per GPU here (each rank reads RANK / WORLD_SIZE as under torchrun)
+        import socket
+        import torch.multiprocessing as mp
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        mp.spawn(_spawned, args=(args, port), nprocs=args.gpus, join=True)
         return
-    if world > 1:
-        pdist.init("nccl", torch.device("cuda", local_rank))
-    try:
-        run_ours(args, rank, world, local_rank)
-    finally:
-        if world > 1:
-            torch.distributed.destroy_process_group()
+    run(args)
 
 
 if __name__ == "__main__":

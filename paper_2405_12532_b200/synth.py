@@ -114,6 +114,28 @@ def uniform_token_ids(batch: int, prompt_len: int, vocab: int, seed: int = 0) ->
     return torch.randint(0, vocab, (batch, prompt_len), generator=gen, dtype=torch.int64)
 
 
+def tiny_llama_weights(hidden: int = 256, n_layers: int = 2, inter: int = 768, vocab: int = 1000, seed: int = 1,
+                       std: float = 0.02) -> dict:
+    """Random-init weights of the tiny Llama-style decoder as fp32 CPU tensors: every matrix
+    N(0, std^2) from one seeded generator in a fixed order, norm gains 1. Matrices are stored
+    [in, out]. Draws values only."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    rn = lambda *shape: torch.randn(*shape, generator=gen, dtype=torch.float32) * std
+    W = {"emb": rn(vocab, hidden)}
+    for l in range(n_layers):
+        for nm in ("wq", "wk", "wv", "wo"):
+            W[f"{nm}{l}"] = rn(hidden, hidden)
+        W[f"wg{l}"] = rn(hidden, inter)
+        W[f"wu{l}"] = rn(hidden, inter)
+        W[f"wd{l}"] = rn(inter, hidden)
+        W[f"n1{l}"] = torch.ones(hidden)
+        W[f"n2{l}"] = torch.ones(hidden)
+    W["nf"] = torch.ones(hidden)
+    W["head"] = rn(hidden, vocab)
+    return W
+
+
 def shard_batch(batch: int, world_size: int, rank: int) -> tuple[int, int]:
     """[start, stop) of the sequences rank `rank` owns when a batch is split
     across data-parallel ranks (sequences are independent: no exchange)."""

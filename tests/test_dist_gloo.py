@@ -54,3 +54,20 @@ def test_two_gloo_ranks_agree_on_time_and_rate():
 def test_single_rank_needs_no_process_group():
     assert pdist.max_over_ranks([1.5, 0.25], 1) == [1.5, 0.25]
     assert pdist.whole_job_rate(64 * 2048, 1, 0.1) == pytest.approx(64 * 2048 / 0.1)
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` outside a launcher starts two ranks itself; its dry run goes through the
+    same rendezvous, barrier and max-over-ranks as the timed run, on gloo, and prints one line."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--dry-run"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["slowest_rank_seconds"] == 2.0 and out["rank0_sequences"] == [0, 64]

@@ -207,6 +207,17 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, c
                              const void* v_new, void* out, void* stream);
 
 /*
+ * (No counterpart in the paper: a test aid for the failure path of the bounded device-side
+ * waits.) Arms the cache so that the NEXT pyr_decode_attn call's loader thread leaves the first
+ * chunk of cache rows of every split out and every wait of that launch spins a few thousand times
+ * at most: the consumers' waits run out, the kernel returns without faulting or hanging,
+ * pyr_cache_status reports PYR_ERR_TIMEOUT and `out` of that call is undefined. The call after it
+ * is normal again; pyr_cache_reset clears the recorded status. Only the CUDA-core decode kernel
+ * (fewer than 4 query heads per KV head, or fp32) honours it.
+ */
+pyr_status_t pyr_cache_arm_wait_test(pyr_cache_t* cache);
+
+/*
  * Section 4.1, Generation Phase, and Algorithm 1's branch for a cache that
  * already holds past PvC: the recent window has slid over the generated tokens,
  * and the layer's PvC is selected again "the same as the prefill phase". The

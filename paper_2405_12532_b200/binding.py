@@ -24,7 +24,7 @@ PYR_FLAG_GEN_RESELECT = 2
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_status_string", "pyr_version", "pyr_launch_count",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
 
@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         L.pyr_select_compact.argtypes = [vp, i32, vp, vp, i64, i64, i64, vp, i64, i64, i64, i64, pi32, vp]
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.pyr_decode_reselect.argtypes = [vp, i32, pi32, pi32, vp]
+        L.pyr_cache_arm_wait_test.argtypes = [vp]
         L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                               C.c_float, vp]
         L.pyr_decode_attn_noalloc_status.argtypes = [vp, pi32]
@@ -270,6 +271,9 @@ class PyrCache:
             C.c_void_p(rows.data_ptr() if rows is not None else None), row_elems, rows_stride_b, rows_stride_n,
             rows_stride_g, C.byref(n_out), C.c_void_p(_stream_ptr(stream))), "pyr_select_compact")
         return n_out.value
+
+    def arm_wait_test(self):
+        _check(lib().pyr_cache_arm_wait_test(self.handle), "pyr_cache_arm_wait_test")
 
     def decode_reselect(self, layer: int, stream=None):
         """pyr_decode_reselect: returns (context rows scored, rows the cache holds afterwards)."""

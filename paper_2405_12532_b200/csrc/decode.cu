@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecodeArgs a) {
   char* kc = static_cast<char*>(a.kc) + ((size_t)b * a.Hkv + g) * a.cap * row_bytes;
   char* vc = static_cast<char*>(a.vc) + ((size_t)b * a.Hkv + g) * a.cap * row_bytes;
   volatile int* abort_flag = &sm.abort_flag;
+  const uint32_t limit = a.spin_limit ? a.spin_limit : kSpinLimit;
 
   if (t == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -118,15 +119,25 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecodeArgs a) {
     // ------------------------------------------------------------ producer
     if (t == kConsumers) {
       bool ok = true;
-      for (int c = 0; c < nchunks && ok; ++c) {
+      int issued = 0;                                  // chunks handed to the copy engine
+      for (int c = 0; c < nchunks && ok; ++c, ++issued) {
         const int st = c % kStages;
-        if (c >= kStages) ok = mbar_wait(&sm.empty[st], ((c / kStages) - 1) & 1, abort_flag, a.status, PYR_ERR_TIMEOUT);
+        if (c >= kStages) ok = mbar_wait_limit(&sm.empty[st], ((c / kStages) - 1) & 1, limit, abort_flag, a.status, PYR_ERR_TIMEOUT);
         if (!ok) break;
+        if (c == a.skip_chunk) continue;               // (test aid) this chunk never arrives
         const int row = start + c * CH;
         const uint32_t bytes = (uint32_t)min(CH, end_cached - row) * row_bytes;
         mbar_expect_tx(&sm.full[st], 2 * bytes);
         bulk_load(sm.k[st], kc + (size_t)row * row_bytes, bytes, &sm.full[st]);
         bulk_load(sm.v[st], vc + (size_t)row * row_bytes, bytes, &sm.full[st]);
+      }
+      if (*abort_flag) {
+        // A wait ran out somewhere in the CTA: nobody may be left to consume the last copies. They
+        // must have landed before the CTA gives its shared memory back, so wait for them here
+        // (bounded, without recording anything more).
+        volatile int none = 0;
+        for (int c = max(issued - kStages, 0); c < issued; ++c)
+          if (c != a.skip_chunk) mbar_wait_limit(&sm.full[c % kStages], (c / kStages) & 1, kSpinLimit, &none, nullptr, 0);
       }
     }
   } else {
@@ -154,7 +165,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(DecodeArgs a) {
     bool ok = true;
     for (int c = 0; c < nchunks && ok; ++c) {
       const int st = c % kStages;
-      ok = mbar_wait(&sm.full[st], (c / kStages) & 1, abort_flag, a.status, PYR_ERR_TIMEOUT);
+      ok = mbar_wait_limit(&sm.full[st], (c / kStages) & 1, limit, abort_flag, a.status, PYR_ERR_TIMEOUT);
       if (!ok) break;
       const int rows_here = min(CH, ncached - c * CH);
       float kf[U][EPL], vf[U][EPL];

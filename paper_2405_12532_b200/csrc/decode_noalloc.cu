@@ -80,6 +80,7 @@ extern "C" pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new
   if (st != PYR_OK) return st;
   a.part_acc = nullptr; a.part_ml = nullptr;
   a.status = status_word;
+  a.spin_limit = 0; a.skip_chunk = -1;
   if (splits > 1) {
     const size_t acc_floats = (size_t)batch * n_q_heads * splits * head_dim;
     const size_t ml_floats = (size_t)batch * n_q_heads * splits * 2;

@@ -4,7 +4,8 @@
 // window, taken over the cache as it is now. Window query i (oldest first) sees
 // the context and the window rows up to its own.
 //
-// CUDA-core kernels for every dtype and head dim: a thread owns one window
+// bf16 with head dim 128 runs on the warp-level tensor-core MMAs (gen_score_mma_kernel below);
+// the CUDA-core kernel serves every other dtype and head dim: a thread owns one window
 // query, keeps it in registers and walks the cache twice - once for the row's
 // log-sum-exp, once for the weighted column sums, which are reduced over the
 // block's 256 queries in a fixed order (warp tree, then warps in order): the
@@ -108,6 +109,177 @@ __global__ void __launch_bounds__(kGenThreads) gen_score_kernel(GenScoreArgs a) 
   }
 }
 
+// ------------------------------------------------------------------ bf16, head dim 128: warp-level MMAs
+// A CTA takes 128 window queries of one (sequence, head): 8 warps x 16 rows, each warp's rows the A
+// operand of m16n8k16 MMAs held in registers for the whole kernel. The cache rows of the KV head
+// stream through shared memory in tiles of 64 (cp.async, two buffers, rows padded to 272 bytes so
+// that ldmatrix meets no bank conflict). Two passes over the cache as in the kernel above: the rows'
+// log-sum-exp on the accumulator fragments first, then w_i 2^(s - lse_i) summed down the columns -
+// within a thread (its two rows), across the warp's eight row groups by a fixed shuffle tree, across
+// the eight warps in order - so the scores are bit-reproducible.
+constexpr int kMq = 128, kMk = 64, kMkStride = 272;
+
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(256) gen_score_mma_kernel(GenScoreArgs a) {
+  constexpr int D = 128;
+  __shared__ __align__(16) uint8_t ktile[2][kMk * kMkStride];
+  __shared__ float wsum[8][kMk];
+  const int bh = blockIdx.x, qt = blockIdx.y;
+  const int b = bh / a.Hq, h = bh % a.Hq;
+  const int g = h / (a.Hq / a.Hkv);
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int gq = lane >> 2, tq = lane & 3;
+  const int c = a.c;
+  const __nv_bfloat16* kbase = static_cast<const __nv_bfloat16*>(a.kc) + ((int64_t)b * a.Hkv + g) * (int64_t)a.cap * D;
+  const float sc2 = a.scale * kLog2e;
+
+  // window rows of this thread: i0 and i0 + 8; A fragments of both for the 8 k-steps
+  const int i0 = qt * kMq + warp * 16 + gq, i1 = i0 + 8;
+  uint32_t qa[8][4];
+  {
+    const __nv_bfloat16* qw = static_cast<const __nv_bfloat16*>(a.qwin);
+    auto qrow = [&](int i) {
+      const int slot = (a.start + i) % a.R;
+      return reinterpret_cast<const uint32_t*>(qw + (((int64_t)b * a.R + slot) * a.Hq + h) * (int64_t)D);
+    };
+    const uint32_t* r0 = qrow(i0 < a.Lw ? i0 : 0);
+    const uint32_t* r1 = qrow(i1 < a.Lw ? i1 : 0);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = i0 < a.Lw ? r0[ks * 8 + tq] : 0u;          // d = 16 ks + 2 tq, + 1
+      qa[ks][1] = i1 < a.Lw ? r1[ks * 8 + tq] : 0u;
+      qa[ks][2] = i0 < a.Lw ? r0[ks * 8 + 4 + tq] : 0u;      // d = 16 ks + 8 + 2 tq, + 1
+      qa[ks][3] = i1 < a.Lw ? r1[ks * 8 + 4 + tq] : 0u;
+    }
+  }
+  const float w0 = i0 < a.Lw ? a.w[i0] : 0.f, w1 = i1 < a.Lw ? a.w[i1] : 0.f;
+  const int last0 = c + i0, last1 = c + i1;           // the newest cache row each query sees
+
+  // ldmatrix: lane supplies row (lane & 7) of matrix (lane >> 3): matrices (keys 0-7, d lo), (keys 0-7, d hi),
+  // (keys 8-15, d lo), (keys 8-15, d hi) of a 16-key, 16-d block
+  const uint32_t lm_off = (uint32_t)(((lane >> 4) * 8 + (lane & 7)) * kMkStride + ((lane >> 3) & 1) * 16);
+
+  auto issue_tile = [&](int j0, int buf) {
+    for (int e = t; e < kMk * 16; e += 256) {
+      const int row = e >> 4, ch = e & 15;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&ktile[buf][row * kMkStride + ch * 16]);
+      if (j0 + row < a.len) cp_async16(dst, kbase + (int64_t)(j0 + row) * D + ch * 8);
+      else *reinterpret_cast<uint4*>(&ktile[buf][row * kMkStride + ch * 16]) = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  // S of this warp's 16 rows x the tile's 64 keys: sc[nb][0,1] = row i0, keys 8 nb + 2 tq (+1); [2,3] = row i1
+  auto tile_scores = [&](int buf, float (*sc)[4]) {
+    const uint32_t kb = (uint32_t)__cvta_generic_to_shared(&ktile[buf][0]) + lm_off;
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+#pragma unroll
+    for (int np = 0; np < 4; ++np) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        uint32_t bf[4];
+        ldsm4(kb + np * 16 * kMkStride + ks * 32, bf);
+        mma16816(sc[2 * np], qa[ks], bf[0], bf[1]);
+        mma16816(sc[2 * np + 1], qa[ks], bf[2], bf[3]);
+      }
+    }
+  };
+
+  // pass 1: log2-domain log-sum-exp of rows i0 and i1 over the cache rows they see
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  const int ntiles = (a.len + kMk - 1) / kMk;
+  issue_tile(0, 0);
+  for (int tI = 0; tI < ntiles; ++tI) {
+    if (tI + 1 < ntiles) issue_tile((tI + 1) * kMk, (tI + 1) & 1);
+    if (tI + 1 < ntiles) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    float sc[8][4];
+    tile_scores(tI & 1, sc);
+    const int j0 = tI * kMk;
+    float x0 = -INFINITY, x1 = -INFINITY;
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int j = j0 + nb * 8 + tq * 2 + e;
+        sc[nb][e] = (j <= last0 && j < a.len) ? sc[nb][e] * sc2 : -INFINITY;
+        sc[nb][2 + e] = (j <= last1 && j < a.len) ? sc[nb][2 + e] * sc2 : -INFINITY;
+        x0 = fmaxf(x0, sc[nb][e]);
+        x1 = fmaxf(x1, sc[nb][2 + e]);
+      }
+    }
+    x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, 1)); x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, 2));
+    x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, 1)); x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, 2));
+    const float n0 = fmaxf(m0, x0), n1 = fmaxf(m1, x1);
+    float s0 = 0.f, s1 = 0.f;
+    if (n0 > -INFINITY) {
+#pragma unroll
+      for (int nb = 0; nb < 8; ++nb) s0 += exp2f(sc[nb][0] - n0) + exp2f(sc[nb][1] - n0);
+      l0 = l0 * exp2f(m0 - n0) + s0;
+      m0 = n0;
+    }
+    if (n1 > -INFINITY) {
+#pragma unroll
+      for (int nb = 0; nb < 8; ++nb) s1 += exp2f(sc[nb][2] - n1) + exp2f(sc[nb][3] - n1);
+      l1 = l1 * exp2f(m1 - n1) + s1;
+      m1 = n1;
+    }
+    __syncthreads();      // the buffer this tile used is refilled two tiles on
+  }
+  // the row sums are spread over the four threads of a row
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float lse0 = m0 + log2f(l0), lse1 = m1 + log2f(l1);
+
+  // pass 2: E[j] = sum_i w_i 2^(s_ij - lse_i) over the CTA's 128 queries, context rows only
+  float* part = a.part + (((int64_t)b * a.Hq + h) * gridDim.y + qt) * (int64_t)c;
+  const int ctiles = (c + kMk - 1) / kMk;
+  issue_tile(0, 0);
+  for (int tI = 0; tI < ctiles; ++tI) {
+    if (tI + 1 < ctiles) issue_tile((tI + 1) * kMk, (tI + 1) & 1);
+    if (tI + 1 < ctiles) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    float sc[8][4];
+    tile_scores(tI & 1, sc);
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        // every context row is visible to every window query
+        float v = w0 * exp2f(sc[nb][e] * sc2 - lse0) + w1 * exp2f(sc[nb][2 + e] * sc2 - lse1);
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (gq == 0) wsum[warp][nb * 8 + tq * 2 + e] = v;
+      }
+    }
+    __syncthreads();
+    const int j0 = tI * kMk;
+    if (t < kMk && j0 + t < c) {
+      float v = 0.f;
+#pragma unroll
+      for (int wI = 0; wI < 8; ++wI) v += wsum[wI][t];
+      part[j0 + t] = v;
+    }
+    // (the next iteration's first barrier separates these reads of wsum from its writes)
+  }
+}
+
 // score[b, g, j] = mean over the query heads of group g of the sum over the
 // window's query tiles of the per-head partial scores, in a fixed order.
 __global__ void __launch_bounds__(256) gen_pool_kernel(GenScoreArgs a, int qtiles) {
@@ -141,13 +313,15 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(const char* src, char* d
 
 }  // namespace
 
-int gen_score_qtiles(int Lw) { return (Lw + kGenThreads - 1) / kGenThreads; }
+// query tiles of the finer-grained of the two kernels: what the per-head partial buffer is sized for
+int gen_score_qtiles(int Lw) { return (Lw + kMq - 1) / kMq; }
 
 cudaError_t launch_gen_score(const GenScoreArgs& a, cudaStream_t s) {
   if (a.c <= 0 || a.Lw <= 0) return cudaSuccess;
-  const int qtiles = gen_score_qtiles(a.Lw);
+  const bool mma = a.dtype == PYR_BF16 && a.D == 128;
+  const int qtiles = mma ? (a.Lw + kMq - 1) / kMq : (a.Lw + kGenThreads - 1) / kGenThreads;
   dim3 grid(a.B * a.Hq, qtiles);
-  if (a.dtype == PYR_BF16 && a.D == 128) gen_score_kernel<__nv_bfloat16, 128><<<grid, kGenThreads, 0, s>>>(a);
+  if (mma) gen_score_mma_kernel<<<grid, 256, 0, s>>>(a);
   else if (a.dtype == PYR_BF16 && a.D == 64) gen_score_kernel<__nv_bfloat16, 64><<<grid, kGenThreads, 0, s>>>(a);
   else if (a.dtype == PYR_F32 && a.D == 128) gen_score_kernel<float, 128><<<grid, kGenThreads, 0, s>>>(a);
   else if (a.dtype == PYR_F32 && a.D == 64) gen_score_kernel<float, 64><<<grid, kGenThreads, 0, s>>>(a);

@@ -148,6 +148,7 @@ struct pyr_cache {
   int last_selected;  // layer of the last pyr_select_compact, -1 if none
   int last_prefilled;
   bool needs_init;
+  bool wait_test_armed;   // pyr_cache_arm_wait_test: the next decode call's loader leaves a chunk out
   float scale;
 };
 
@@ -239,6 +240,7 @@ pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t byte
   c->q_count.assign(cfg->n_layers, 0);
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
   c->needs_init = true;
+  c->wait_test_armed = false;
   c->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
   } catch (...) {           // the host-side vectors could not be allocated
     delete c;
@@ -456,6 +458,9 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   a.len = c->len_now[layer]; a.cap = p.cap;
   a.scale = c->scale; a.dtype = c->cfg.dtype;
   a.status = at<int>(c, c->lay.status);
+  a.spin_limit = c->wait_test_armed ? 4096u : 0u;
+  a.skip_chunk = c->wait_test_armed ? 0 : -1;
+  c->wait_test_armed = false;
   int splits = 1, rps = 0;
   const int sms = pyr::device_sm_count();
   if (sms <= 0) return PYR_ERR_CUDA;
@@ -475,6 +480,12 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
     g_launches += 1;
     c->q_count[layer] += 1;
   }
+  return PYR_OK;
+}
+
+pyr_status_t pyr_cache_arm_wait_test(pyr_cache_t* c) {
+  if (!c) return PYR_ERR_NULL;
+  c->wait_test_armed = true;
   return PYR_OK;
 }
 

@@ -69,6 +69,8 @@ struct DecodeArgs {
   float scale;
   int dtype;
   int* status;                     // device status word, may be null
+  uint32_t spin_limit = 0;         // iterations a device-side wait may spin; 0 = the default
+  int skip_chunk = -1;                // -1; else the loader leaves this chunk of every split out (exercises the waits' failure path)
 };
 
 // Split-K rule of the decode kernels: rows [0, total) of a cache are cut into `splits` ranges of

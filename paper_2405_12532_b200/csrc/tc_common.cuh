@@ -49,15 +49,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // the global status word, and returns false.
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, uint32_t limit, volatile int* abort_flag,
+                                                int* status, int code) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
   *abort_flag = 1;
   if (status) atomicCAS(status, 0, code);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+  return mbar_wait_limit(bar, parity, kSpinLimit, abort_flag, status, code);
 }
 
 // ---------------------------------------------------------------- TMA

@@ -71,6 +71,9 @@ typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
 
 /* flags */
 #define PYR_FLAG_CUDA_CORE_PREFILL 1u /* bf16 prefill on the CUDA-core kernel (validation aid) */
+#define PYR_FLAG_POS_REENCODE 4u      /* Appendix A.2, first choice: the kept tokens' positions are re-encoded from 0
+                                         in order after every selection; default is the second choice (gather the
+                                         original positions), which the paper finds slightly better */
 #define PYR_FLAG_GEN_RESELECT 2u      /* keep each layer's recent queries so that pyr_decode_reselect can
                                          update the PvC during generation (Section 4.1, Generation Phase) */
 
@@ -83,7 +86,9 @@ typedef struct {
   int32_t n_layers;
   int32_t n_q_heads;      /* Hq                                                        */
   int32_t n_kv_heads;     /* Hkv, divides Hq                                           */
-  int32_t head_dim;       /* D: 64 or 128                                              */
+  int32_t head_dim;       /* D: 64 or 128. The tensor-core (tcgen05) prefill kernels are
+                             built for bf16 with D = 128; bf16 with D = 64 and all of fp32
+                             run on the CUDA-core kernels, far below tensor-core speed     */
   int32_t sel_groups;     /* G: 1 (one kept set per sequence) or Hkv (one per KV head) */
   int32_t dtype;          /* pyr_dtype_t of q/k/v/out and of the cache                 */
   int32_t batch;          /* B                                                         */
@@ -94,7 +99,12 @@ typedef struct {
                              c_0 = N - L that layer l keeps; each in [0,1],
                              non-increasing                                            */
   const int32_t* min_len; /* host [n_layers] or NULL: N_l, lower bound on the kept
-                             length (window included) of layer l                       */
+                             length (window included) of layer l. FIXED-COUNT MODE
+                             (Section 4.1, last sentence: a fixed number of PvCs per layer,
+                             "unlimited input like StreamingLLM"): ratio[l] = 0 and
+                             min_len[l] = count_l + L keep exactly count_l context keys in
+                             layer l; with pyr_decode_reselect every s <= T steps the cache
+                             never exceeds count_l + L + s rows however long the generation */
   const float* recent_w;  /* host [L] or NULL: non-negative weights of the recent
                              queries, oldest first. NULL = linear ramp
                              2(i+1)/(L(L+1)), which sums to 1                          */
@@ -205,6 +215,12 @@ pyr_status_t pyr_select_compact(pyr_cache_t* cache, int32_t layer, const void* k
  */
 pyr_status_t pyr_decode_attn(pyr_cache_t* cache, int32_t layer, const void* q, const void* k_new,
                              const void* v_new, void* out, void* stream);
+
+/* Section 5.2, "Recent Sequence Ratio": the recent sequence S_r given as a fraction of the input
+ * (the paper settles on 40 %). Returns the window length for pyr_config_t.recent_len:
+ * floor(ratio * prompt_len) clamped to [1, prompt_len]; 0 for a negative ratio or an empty prompt.
+ * Host arithmetic only. */
+int32_t pyr_recent_len_from_ratio(int32_t prompt_len, double ratio);
 
 /*
  * (No counterpart in the paper: a test aid for the failure path of the bounded device-side

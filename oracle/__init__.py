@@ -8,6 +8,7 @@ its only callers.
 from .pyramid import (  # noqa: F401
     softmax_scale_default,
     recent_weights,
+    recent_len_from_ratio,
     layer_budgets,
     attention_weights,
     causal_attention,

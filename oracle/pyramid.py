@@ -53,6 +53,15 @@ def recent_weights(L: int) -> np.ndarray:
     return 2.0 * (i + 1.0) / (F64(L) * F64(L + 1))
 
 
+def recent_len_from_ratio(prompt_len: int, ratio: float) -> int:
+    """Section 5.2, "Recent Sequence Ratio": the window as a fraction of the input.
+    L = floor(ratio * N) clamped to [1, N]; 0 for a negative ratio or an empty prompt."""
+    N = int(prompt_len)
+    if N < 1 or not ratio >= 0:
+        return 0
+    return int(min(N, max(1, np.floor(F64(ratio) * F64(N)))))
+
+
 def layer_budgets(prompt_len: int, recent_len: int, ratio, min_len=None):
     """Per-layer sizes of the pyramid (Algorithm 1: ratio p, its decay, the
     minimum PvC lengths N_l; Section 4.1).
@@ -172,7 +181,7 @@ def gather_rows(x: np.ndarray, kept: np.ndarray, axis: int = 0) -> np.ndarray:
 
 
 def prefill_layer(Q, K, V, recent_len: int, k_keep: int, sel_groups: int,
-                  scale: float | None = None, w=None, pos=None, out_rows=None):
+                  scale: float | None = None, w=None, pos=None, out_rows=None, reencode: bool = False):
     """One layer of Algorithm 1's prefill branch on a batch.
 
     Q [B, n, Hq, D], K/V [B, n, Hkv, D] are the layer's inputs for the n tokens
@@ -228,7 +237,8 @@ def prefill_layer(Q, K, V, recent_len: int, k_keep: int, sel_groups: int,
             Kk[b, g] = gather_rows(K[b, :, g], idx)
             Vk[b, g] = gather_rows(V[b, :, g], idx)
         for gg in range(G):
-            pk[b, gg] = gather_rows(pos[b, gg], kept[b, gg])
+            # Appendix A.2: gather the original positions (default), or re-encode from 0 in order
+            pk[b, gg] = np.arange(n_out) if reencode else gather_rows(pos[b, gg], kept[b, gg])
     return {"O": np.stack(Os), "lse": np.stack(lses), "score": np.stack(scores),
             "kept": kept, "K_kept": Kk, "V_kept": Vk, "pos_kept": pk}
 

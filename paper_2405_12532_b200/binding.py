@@ -20,11 +20,12 @@ PYR_ERR_HOST_MEMORY = 10
 PYR_BF16, PYR_F32 = 0, 1
 PYR_FLAG_CUDA_CORE_PREFILL = 1
 PYR_FLAG_GEN_RESELECT = 2
+PYR_FLAG_POS_REENCODE = 4
 
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_status_string", "pyr_version", "pyr_launch_count",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
 
@@ -80,12 +81,14 @@ def lib() -> C.CDLL:
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.pyr_decode_reselect.argtypes = [vp, i32, pi32, pi32, vp]
         L.pyr_cache_arm_wait_test.argtypes = [vp]
+        L.pyr_recent_len_from_ratio.argtypes = [i32, C.c_double]
+        L.pyr_recent_len_from_ratio.restype = i32
         L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
                                               C.c_float, vp]
         L.pyr_decode_attn_noalloc_status.argtypes = [vp, pi32]
         for name in EXPORTS:
             fn = getattr(L, name)
-            if name not in ("pyr_status_string", "pyr_version", "pyr_launch_count"):
+            if name not in ("pyr_status_string", "pyr_version", "pyr_launch_count", "pyr_recent_len_from_ratio"):
                 fn.restype = C.c_int
         _lib = L
     return _lib
@@ -154,6 +157,10 @@ def decode_attn_noalloc(q, k_new, v_new, out, k_cache, v_cache, length: int, sof
     return lib().pyr_decode_attn_noalloc(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                          k_cache.data_ptr(), v_cache.data_ptr(), B, Hq, Hkv, D, dt, int(length),
                                          cap, float(softmax_scale), C.c_void_p(_stream_ptr(stream)))
+
+
+def recent_len_from_ratio(prompt_len: int, ratio: float) -> int:
+    return int(lib().pyr_recent_len_from_ratio(int(prompt_len), float(ratio)))
 
 
 def decode_attn_noalloc_status(stream=None) -> int:

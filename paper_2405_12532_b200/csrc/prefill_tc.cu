@@ -140,7 +140,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     return it;
   };
   volatile int* abort_flag = &sm.abort_flag;
-  if (*reinterpret_cast<volatile int*>(a.status) != 0) return;   // an earlier CTA gave up: do not pile on
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
@@ -153,9 +152,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(&sm.s_full[i], 1);
       mbar_init(&sm.s_empty[i], kTile);          // the group that reads the buffer
     }
-    sm.abort_flag = 0;
+    // an earlier CTA of this launch gave up: the whole CTA leaves together (decided by one thread)
+    sm.abort_flag = *reinterpret_cast<volatile int*>(a.status) != 0 ? 2 : 0;
     fence_barrier_init();
   }
+  __syncthreads();
+  if (sm.abort_flag == 2) return;
   if (warp == kScoreCompute) {
     tmem_alloc(&sm.tmem_base, kScoreBufs * kTile);
     tmem_relinquish();

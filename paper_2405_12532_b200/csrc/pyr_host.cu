@@ -410,6 +410,7 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
   sa.pos_in = layer == 0 ? nullptr : pos_in;
   sa.pos_out = pos_out;
   sa.B = c->cfg.batch; sa.G = c->cfg.sel_groups; sa.n = p.n_in; sa.c = p.c; sa.k = p.k;
+  sa.reencode = (c->cfg.flags & PYR_FLAG_POS_REENCODE) ? 1 : 0;
   if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
 
   pyr::GatherArgs ga;
@@ -481,6 +482,14 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
     c->q_count[layer] += 1;
   }
   return PYR_OK;
+}
+
+int32_t pyr_recent_len_from_ratio(int32_t prompt_len, double ratio) {
+  if (prompt_len < 1 || !(ratio >= 0.0)) return 0;
+  long long L = (long long)std::floor(ratio * (double)prompt_len);
+  if (L < 1) L = 1;
+  if (L > prompt_len) L = prompt_len;
+  return (int32_t)L;
 }
 
 pyr_status_t pyr_cache_arm_wait_test(pyr_cache_t* c) {

@@ -30,6 +30,7 @@ struct SelectArgs {
   const int32_t* pos_in;   // [B, G, n] or nullptr = identity
   int32_t* pos_out;    // [B, G, n_out]
   int B, G, n, c, k;   // n_out = k + (n - c)
+  int reencode = 0;    // 1: positions are re-encoded from 0 in kept order instead of gathered
 };
 
 struct GatherArgs {

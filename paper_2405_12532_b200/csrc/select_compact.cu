@@ -38,13 +38,13 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
   // the window is always kept
   for (int i = t; i < window; i += kSelThreads) {
     idx[k + i] = c + i;
-    pos_out[k + i] = pos_in ? pos_in[c + i] : c + i;
+    pos_out[k + i] = a.reencode ? k + i : (pos_in ? pos_in[c + i] : c + i);
   }
   if (k == 0) return;
   if (k == c) {
     for (int i = t; i < c; i += kSelThreads) {
       idx[i] = i;
-      pos_out[i] = pos_in ? pos_in[i] : i;
+      pos_out[i] = a.reencode ? i : (pos_in ? pos_in[i] : i);
     }
     return;
   }
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
     if (keep) {
       const uint32_t p = gt_before + min(eq_before, need_eq);
       idx[p] = i;
-      pos_out[p] = pos_in ? pos_in[i] : i;
+      pos_out[p] = a.reencode ? (int)p : (pos_in ? pos_in[i] : i);
     }
     __syncthreads();
     if (t == kSelThreads - 1) sh_running = before + (gt ? (1u << 16) : 0u) + (eq ? 1u : 0u);

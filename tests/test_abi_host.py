@@ -141,3 +141,11 @@ def test_shard_batch_covers_batch():
         spans = [synth.shard_batch(B, W, r) for r in range(W)]
         assert spans[0][0] == 0 and spans[-1][1] == B
         assert all(spans[i][1] == spans[i + 1][0] for i in range(W - 1))
+
+
+def test_recent_len_from_ratio_matches_the_oracle():
+    for N in (1, 7, 512, 2048, 8191):
+        for r in (0.0, 0.001, 0.3, 0.4, 0.5, 0.9999, 1.0, 1.7):
+            assert pb.recent_len_from_ratio(N, r) == oracle.recent_len_from_ratio(N, r)
+    assert pb.recent_len_from_ratio(2048, 0.4) == 819 and pb.recent_len_from_ratio(10, 0.0) == 1
+    assert pb.recent_len_from_ratio(0, 0.4) == 0 and pb.recent_len_from_ratio(100, -0.1) == 0

@@ -31,6 +31,18 @@ CONFIGS = {
                           dtype="bf16", batch=16, prompt_len=8192, recent_len=1024,
                           ratio=(1.0, 0.2), sel_groups=8, max_new_tokens=512,
                           hitter_frac=0.01, hitter_mag=4.0),
+    # The shapes of the paper's efficiency tables (Table 1 / Table 2: LLaMA-2-13B at batch 32 with
+    # 512 prompt + 256 generated tokens, LLaMA-2-70B at batch 8 with 256 + 128), as attention stacks.
+    # The paper's text does not give the schedule or the window behind its numbers: the window is
+    # 40 % of the prompt (its Section 5.2 trade-off) and the retention falls geometrically to 0.2.
+    "13b_table_32x512": dict(kind="stack", n_layers=40, n_q_heads=40, n_kv_heads=40, head_dim=128,
+                             dtype="bf16", batch=32, prompt_len=512, recent_len=204,
+                             ratio=(1.0, 0.2), sel_groups=40, max_new_tokens=256,
+                             hitter_frac=0.02, hitter_mag=3.0),
+    "70b_table_8x256": dict(kind="stack", n_layers=80, n_q_heads=64, n_kv_heads=8, head_dim=128,
+                            dtype="bf16", batch=8, prompt_len=256, recent_len=102,
+                            ratio=(1.0, 0.2), sel_groups=8, max_new_tokens=128,
+                            hitter_frac=0.01, hitter_mag=4.0),
 }
 
 

@@ -149,3 +149,34 @@ def test_recent_len_from_ratio_matches_the_oracle():
             assert pb.recent_len_from_ratio(N, r) == oracle.recent_len_from_ratio(N, r)
     assert pb.recent_len_from_ratio(2048, 0.4) == 819 and pb.recent_len_from_ratio(10, 0.0) == 1
     assert pb.recent_len_from_ratio(0, 0.4) == 0 and pb.recent_len_from_ratio(100, -0.1) == 0
+
+
+def _cache_gb(w, ratio, batch, flags=0):
+    cfg, keep = pb.make_config(**pb.config_from_workload(dict(w, batch=batch), ratio, flags=flags))
+    return pb.pyr_cache_bytes(cfg)[0] / 1e9
+
+
+def test_max_batch_under_a_memory_cap_table2_shape():
+    """Table 2's setting as byte accounting: the largest batch whose cache buffer fits beside the
+    13B model's 26 GB of 2-byte weights on an 80 GB device, with every layer keeping everything and
+    with the pyramid schedule (no GPU: pyr_cache_bytes is host arithmetic). The paper reports batch
+    42 for the full cache and 88 for PyramidInfer, a factor 2.1; its schedule is not in its text, so
+    only the direction and rough size of the gain are checked."""
+    w = synth.CONFIGS["13b_table_32x512"]
+    budget_gb = 80.0 - 26.0
+
+    def max_batch(ratio, generated_rows):
+        lo, hi = 1, 4096
+        while lo < hi:
+            mid = (lo + hi + 1) // 2
+            if _cache_gb(dict(w, max_new_tokens=generated_rows), ratio, mid) <= budget_gb:
+                lo = mid
+            else:
+                hi = mid - 1
+        return lo
+
+    full = max_batch([1.0] * w["n_layers"], 256)
+    # with the generation-phase update every 16 steps a layer never holds more than its budget + window + 16 rows
+    pyr = max_batch(synth.ratio_schedule(w), 16)
+    assert 60 <= full <= 90             # 2 * 40 layers * 5120 * 2 B * 768 rows = 0.63 GB per sequence
+    assert pyr / full > 1.8

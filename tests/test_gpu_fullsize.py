@@ -23,6 +23,9 @@ CASES = [
     ("7b_64x2k", [0, 6, 12, 19, 26, 31], 6),
     ("13b_stack_32x4k", [0, 7, 15, 23, 31, 39], 6),
     ("70b_gqa_16x8k", [0, 16, 32, 48, 64, 79], 4),
+    # the shapes of the paper's efficiency tables (short prompts: every layer is memory-bound)
+    ("13b_table_32x512", [0, 13, 26, 39], 6),
+    ("70b_table_8x256", [0, 40, 79], 4),
 ]
 
 

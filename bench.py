@@ -327,11 +327,12 @@ def run_ours(args, rank, world, local_rank, workload=None):
                                 "capture at batch 16 by the Q+K+V+O bytes",
                 "peak_source": f"of {peak_src}", "launches": K * nL * 2, "avg_layer_us": t_attn / (K * nL) * 1e6}
     ach_sel = K * wl.select_compact_bytes() / t_sel / 1e9
-    rr = traffic_ratio("gather_kv_kernel_7b_2k_batch16.txt")
+    rr = traffic_ratio("select_compact_7b_2k_batch16.txt")
     roof_sel = {"kernel": "select + gather + compact", "bound": "hbm", "achieved": ach_sel, "peak": hbm,
                 "unit": "GB/s", "frac": ach_sel / hbm,
                 "traffic": rr * wl.select_compact_bytes() / nL if rr else None,
-                "traffic_note": "dram bytes per layer, scaled from the gather kernel's ncu capture at batch 16",
+                "traffic_note": "dram bytes per layer (average), scaled from the ncu captures of the call's three kernels at "
+                                "batch 16 (profiles/select_compact_7b_2k_batch16.txt)",
                 "peak_source": f"of {peak_src}", "avg_layer_us": t_sel / (K * nL) * 1e6}
     dominant = roof_dec if (roof_dec and t_dec >= t_attn) else roof_pre
     line = {

@@ -309,6 +309,35 @@ pyr_status_t pyr_decode_attn_noalloc(const void* q, const void* k_new, const voi
  */
 pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
 
+/*
+ * Decoder glue for whole-model workloads. (No counterpart in the paper beyond Appendix A.2's
+ * choice of positions: these are the public Llama block's steps around the pyramid path, so that a
+ * model can run end to end on this library's kernels. CUDA-core kernels, fp32 arithmetic, for fp32
+ * or bf16 storage; dtype is a pyr_dtype_t.) All pointers are device pointers, tensors row-major and
+ * contiguous, every call asynchronous on `stream`.
+ *   embed   out[t, :] = table[ids[t], :]; table [vocab, d]. An id outside [0, vocab) zeroes its row
+ *           and, if dev_status (a device int, may be NULL) is given, records PYR_ERR_INVALID in it.
+ *   rmsnorm out = x / sqrt(mean(x^2) + eps) * gain; x, out [tokens, d] (may alias), gain [d].
+ *   linear  y[m, n] = x[m, k] . w[n, k] (+ residual[m, n] if not NULL); w is [n, k] ("out, in").
+ *           y may alias residual, not x.
+ *   rope    rotates, in place, the pairs (i, i + head_dim/2) of every head of x [tokens, n_heads,
+ *           head_dim] by pos[t] * 10000^(-2i/head_dim): Appendix A.2's "gather" when pos holds the
+ *           tokens' original positions (pyr_cache_kept's second pointer), "re-encode" when it counts
+ *           from 0.
+ *   swiglu  out = silu(gate) * up, n elements.
+ *   argmax  out[r] = index of the largest of x[r, 0..n), the lowest index on ties; x [rows, n].
+ */
+pyr_status_t pyr_glue_embed(const int32_t* ids, const void* table, void* out, int64_t tokens, int32_t d, int32_t vocab,
+                            int32_t dtype, int32_t* dev_status, void* stream);
+pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int32_t d, float eps,
+                              int32_t dtype, void* stream);
+pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual, void* y, int64_t m, int32_t n,
+                             int32_t k, int32_t dtype, void* stream);
+pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,
+                           int32_t dtype, void* stream);
+pyr_status_t pyr_glue_swiglu(const void* gate, const void* up, void* out, int64_t n, int32_t dtype, void* stream);
+pyr_status_t pyr_glue_argmax(const void* x, int32_t* out, int64_t rows, int32_t n, int32_t dtype, void* stream);
+
 const char* pyr_status_string(pyr_status_t status);
 
 /* Number of kernels this process has launched through the library so far. */

@@ -25,7 +25,8 @@ PYR_FLAG_POS_REENCODE = 4
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_status_string", "pyr_version", "pyr_launch_count",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear",
+    "pyr_glue_rope", "pyr_glue_swiglu", "pyr_glue_argmax", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
 
@@ -81,6 +82,12 @@ def lib() -> C.CDLL:
         L.pyr_decode_attn.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.pyr_decode_reselect.argtypes = [vp, i32, pi32, pi32, vp]
         L.pyr_cache_arm_wait_test.argtypes = [vp]
+        L.pyr_glue_embed.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, vp]
+        L.pyr_glue_rmsnorm.argtypes = [vp, vp, vp, i64, i32, C.c_float, i32, vp]
+        L.pyr_glue_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
+        L.pyr_glue_rope.argtypes = [vp, vp, i64, i32, i32, i32, vp]
+        L.pyr_glue_swiglu.argtypes = [vp, vp, vp, i64, i32, vp]
+        L.pyr_glue_argmax.argtypes = [vp, vp, i64, i32, i32, vp]
         L.pyr_recent_len_from_ratio.argtypes = [i32, C.c_double]
         L.pyr_recent_len_from_ratio.restype = i32
         L.pyr_decode_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
@@ -157,6 +164,61 @@ def decode_attn_noalloc(q, k_new, v_new, out, k_cache, v_cache, length: int, sof
     return lib().pyr_decode_attn_noalloc(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                          k_cache.data_ptr(), v_cache.data_ptr(), B, Hq, Hkv, D, dt, int(length),
                                          cap, float(softmax_scale), C.c_void_p(_stream_ptr(stream)))
+
+
+def _dt(t: torch.Tensor) -> int:
+    return PYR_BF16 if t.dtype == torch.bfloat16 else PYR_F32
+
+
+def glue_embed(ids, table):
+    """ids int32 [...], table [V, d] -> [..., d] (pyr_glue_embed)."""
+    assert ids.dtype == torch.int32 and ids.is_contiguous() and table.is_contiguous()
+    out = torch.empty(*ids.shape, table.shape[1], dtype=table.dtype, device=table.device)
+    _check(lib().pyr_glue_embed(ids.data_ptr(), table.data_ptr(), out.data_ptr(), ids.numel(), table.shape[1],
+                                table.shape[0], _dt(table), None, C.c_void_p(_stream_ptr(None))), "pyr_glue_embed")
+    return out
+
+
+def glue_rmsnorm(x, gain, eps=1e-5):
+    assert x.is_contiguous()
+    out = torch.empty_like(x)
+    _check(lib().pyr_glue_rmsnorm(x.data_ptr(), gain.data_ptr(), out.data_ptr(), x.numel() // x.shape[-1], x.shape[-1],
+                                  float(eps), _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_rmsnorm")
+    return out
+
+
+def glue_linear(x, w, residual=None):
+    """x [..., K] . w [N, K] (+ residual [..., N]) -> [..., N] (pyr_glue_linear)."""
+    assert x.is_contiguous() and w.is_contiguous() and (residual is None or residual.is_contiguous())
+    N, K = w.shape
+    y = torch.empty(*x.shape[:-1], N, dtype=x.dtype, device=x.device)
+    _check(lib().pyr_glue_linear(x.data_ptr(), w.data_ptr(), residual.data_ptr() if residual is not None else None,
+                                 y.data_ptr(), x.numel() // K, N, K, _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_linear")
+    return y
+
+
+def glue_rope_(x, pos):
+    """In place on x [..., H, D] with pos int32 [...] (pyr_glue_rope)."""
+    assert x.is_contiguous() and pos.dtype == torch.int32 and pos.is_contiguous()
+    _check(lib().pyr_glue_rope(x.data_ptr(), pos.data_ptr(), pos.numel(), x.shape[-2], x.shape[-1], _dt(x),
+                               C.c_void_p(_stream_ptr(None))), "pyr_glue_rope")
+    return x
+
+
+def glue_swiglu(gate, up):
+    assert gate.is_contiguous() and up.is_contiguous()
+    out = torch.empty_like(gate)
+    _check(lib().pyr_glue_swiglu(gate.data_ptr(), up.data_ptr(), out.data_ptr(), gate.numel(), _dt(gate),
+                                 C.c_void_p(_stream_ptr(None))), "pyr_glue_swiglu")
+    return out
+
+
+def glue_argmax(x):
+    assert x.is_contiguous() and x.dim() == 2
+    out = torch.empty(x.shape[0], dtype=torch.int32, device=x.device)
+    _check(lib().pyr_glue_argmax(x.data_ptr(), out.data_ptr(), x.shape[0], x.shape[1], _dt(x),
+                                 C.c_void_p(_stream_ptr(None))), "pyr_glue_argmax")
+    return out
 
 
 def recent_len_from_ratio(prompt_len: int, ratio: float) -> int:

@@ -484,6 +484,49 @@ pyr_status_t pyr_decode_attn(pyr_cache_t* c, int32_t layer, const void* q, const
   return PYR_OK;
 }
 
+// ---- decoder glue of whole-model workloads: argument checks and dispatch
+static bool glue_ok(int32_t dtype, std::initializer_list<const void*> ptrs) {
+  if (dtype != PYR_BF16 && dtype != PYR_F32) return false;
+  for (const void* p : ptrs) if (!p) return false;
+  return true;
+}
+#define PYR_GLUE(call) do { if ((call) != cudaSuccess) return PYR_ERR_CUDA; g_launches += 1; return PYR_OK; } while (0)
+
+pyr_status_t pyr_glue_embed(const int32_t* ids, const void* table, void* out, int64_t tokens, int32_t d, int32_t vocab,
+                            int32_t dtype, int32_t* dev_status, void* stream) {
+  if (!glue_ok(dtype, {ids, table, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (tokens < 0 || d < 1 || vocab < 1) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_embed(ids, table, out, tokens, d, vocab, dtype, dev_status, static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int32_t d, float eps,
+                              int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, gain, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (tokens < 0 || d < 1 || !(eps >= 0.f)) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_rmsnorm(x, gain, out, tokens, d, eps, dtype, static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual, void* y, int64_t m, int32_t n,
+                             int32_t k, int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, w, y})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,
+                           int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, pos})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (tokens < 0 || n_heads < 1 || head_dim < 2 || head_dim % 2) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_rope(x, pos, tokens, n_heads, head_dim, dtype, static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_swiglu(const void* gate, const void* up, void* out, int64_t n, int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {gate, up, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (n < 0) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_swiglu(gate, up, out, n, dtype, static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_argmax(const void* x, int32_t* out, int64_t rows, int32_t n, int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (rows < 0 || n < 1) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_argmax(x, out, rows, n, dtype, static_cast<cudaStream_t>(stream)));
+}
+
 int32_t pyr_recent_len_from_ratio(int32_t prompt_len, double ratio) {
   if (prompt_len < 1 || !(ratio >= 0.0)) return 0;
   long long L = (long long)std::floor(ratio * (double)prompt_len);

@@ -109,6 +109,16 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_gather_kv(const GatherArgs& a, cudaStream_t s);
 cudaError_t launch_compact_rows(const RowsArgs& a, cudaStream_t s);
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s);
+// decoder glue of whole-model workloads (csrc/glue.cu); matrices row-major, w is [N, K] (out, in)
+cudaError_t launch_glue_embed(const int32_t* ids, const void* table, void* out, int64_t tokens, int d, int vocab,
+                              int dtype, int* status, cudaStream_t s);
+cudaError_t launch_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int d, float eps, int dtype,
+                                cudaStream_t s);
+cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int dtype,
+                               cudaStream_t s);
+cudaError_t launch_glue_rope(void* x, const int32_t* pos, int64_t tokens, int H, int D, int dtype, cudaStream_t s);
+cudaError_t launch_glue_swiglu(const void* g, const void* u, void* out, int64_t n, int dtype, cudaStream_t s);
+cudaError_t launch_glue_argmax(const void* x, int32_t* out, int64_t rows, int n, int dtype, cudaStream_t s);
 int gen_score_qtiles(int Lw);
 cudaError_t launch_gen_score(const GenScoreArgs& a, cudaStream_t s);     // two kernels
 // rows of row_bytes (a multiple of 16) per batch entry, byte strides

@@ -1,0 +1,154 @@
+"""The 7B Llama-shaped workload as a whole model on the library's kernels, at batch 1: 32 layers, hidden
+4096, 32 heads x 128, MLP 11008, vocabulary 32000, bf16, random-init weights (seed 1), uniform random token
+ids (seed 0), prompt 2048, window 256, the geometric schedule 1.0 -> 0.3, one kept set per sequence, then
+two decode steps. An fp64 run of this size is out of reach, and a bf16 chain of 32 layers is only
+meaningful per call, so every call is checked on the inputs the GPU call had: sampled outputs of the
+linear layers, norms and rotary embedding against fp64 formulas, attention rows, scores and kept sets of
+sampled layers against the oracle, the hidden-row compaction byte for byte."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import tiny_llama as tl
+from paper_2405_12532_b200 import binding as pb
+from paper_2405_12532_b200 import synth
+from parity_util import check_kept
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+NL, HID, H, D, FF, V, N, L, B, T = 32, 4096, 32, 128, 11008, 32000, 2048, 256, 1, 2
+
+
+def _weights():
+    g = torch.Generator(device=DEV)
+    g.manual_seed(1)
+    rn = lambda *s: (torch.randn(*s, generator=g, device=DEV, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    W = {"emb": rn(V, HID), "head": rn(V, HID), "nf": torch.ones(HID, device=DEV, dtype=torch.bfloat16)}
+    for l in range(NL):
+        for nm, shape in (("wq", (HID, HID)), ("wk", (HID, HID)), ("wv", (HID, HID)), ("wo", (HID, HID)),
+                          ("wg", (FF, HID)), ("wu", (FF, HID)), ("wd", (HID, FF))):
+            W[f"{nm}{l}"] = rn(*shape)                                   # [out, in]
+        W[f"n1{l}"] = torch.ones(HID, device=DEV, dtype=torch.bfloat16)
+        W[f"n2{l}"] = torch.ones(HID, device=DEV, dtype=torch.bfloat16)
+    return W
+
+
+def _check_linear(x, w, y, rng, res=None, count=24):
+    """Sampled entries of y = x w^T (+ res) against fp64 dot products of the bf16 inputs."""
+    M, Nn = y.shape[-2], y.shape[-1]
+    x2, y2 = x.reshape(-1, x.shape[-1]), y.reshape(-1, Nn)
+    r2 = None if res is None else res.reshape(-1, Nn)
+    rows = torch.from_numpy(rng.integers(0, x2.shape[0], size=count)).to(DEV)
+    cols = torch.from_numpy(rng.integers(0, Nn, size=count)).to(DEV)
+    want = (x2[rows].double() * w[cols].double()).sum(-1)
+    if r2 is not None:
+        want = want + r2[rows, cols].double()
+    got = y2[rows, cols].double()
+    scale = float(want.abs().max().clamp_min(1e-3))
+    assert float((got - want).abs().max()) <= 2 ** -7 * scale + 1e-4, (float((got - want).abs().max()), scale)
+
+
+def test_7b_shaped_model_batch1_all_layers():
+    W = _weights()
+    rng = np.random.default_rng(5)
+    w = dict(synth.CONFIGS["7b_64x2k"], batch=B, max_new_tokens=T)
+    ratio = synth.ratio_schedule(w)
+    budgets = oracle.layer_budgets(N, L, ratio)
+    cache = pb.PyrCache(device=DEV, **pb.config_from_workload(w, ratio))
+    ids = synth.uniform_token_ids(B, N, V, seed=0).to(torch.int32).to(DEV)
+    x = pb.glue_embed(ids, W["emb"])
+    assert torch.equal(x[0, 7], W["emb"][int(ids[0, 7])])
+    pos = torch.arange(N, device=DEV, dtype=torch.int32).expand(B, N).contiguous()
+    wts = oracle.recent_weights(L)
+    checked = [0, 9, 19, 31]
+    exact = ties = 0
+    for l, bud in enumerate(budgets):
+        n, c, k = bud["n_in"], bud["c"], bud["k"]
+        assert x.shape[1] == n == cache.layer_info(l)["n_in"]
+        h = pb.glue_rmsnorm(x, W[f"n1{l}"])
+        q = pb.glue_linear(h, W[f"wq{l}"]).view(B, n, H, D)
+        kk = pb.glue_linear(h, W[f"wk{l}"]).view(B, n, H, D)
+        v = pb.glue_linear(h, W[f"wv{l}"]).view(B, n, H, D)
+        if l in checked:
+            r = int(rng.integers(n))
+            np.testing.assert_allclose(synth.widen(h[0, r]), tl.rmsnorm(synth.widen(x[0, r]), 1.0), rtol=2 ** -7, atol=1e-3)
+            _check_linear(h, W[f"wq{l}"], q.view(B, n, HID), rng)
+            _check_linear(h, W[f"wv{l}"], v.view(B, n, HID), rng)
+            q0 = q.clone()
+        pb.glue_rope_(q, pos)
+        pb.glue_rope_(kk, pos)
+        if l in checked:
+            rows = rng.integers(0, n, size=4)
+            want = tl.rope(synth.widen(q0[0, rows]), pos[0, rows].cpu().numpy())
+            assert np.abs(synth.widen(q[0, rows]) - want).max() <= 2 ** -7 * np.abs(want).max()
+        o = torch.empty_like(q)
+        cache.prefill_layer(l, q, kk, v, o)
+        if l in checked:
+            torch.cuda.synchronize()
+            score = cache.scores(l).clone()
+            E = np.zeros((H, c))
+            for hh in range(H):
+                A, _ = oracle.attention_weights(synth.widen(q[0, :, hh]), synth.widen(kk[0, :, hh]),
+                                                oracle.softmax_scale_default(D), np.arange(c, n))
+                E[hh] = oracle.ensemble_score(A, L, wts)
+            sc_ref = E.mean(0)
+            np.testing.assert_allclose(synth.widen(score[0, 0]), sc_ref, rtol=2e-3, atol=1e-30)
+            hh = int(rng.integers(H))
+            rs = np.sort(rng.choice(n, size=32, replace=False)); rs[-1] = n - 1
+            A, _ = oracle.attention_weights(synth.widen(q[0, :, hh]), synth.widen(kk[0, :, hh]),
+                                            oracle.softmax_scale_default(D), rs)
+            assert np.abs(synth.widen(o[0, torch.from_numpy(rs).to(DEV), hh]) - A @ synth.widen(v[0, :, hh])).max() <= 2e-2
+        rows_t = torch.cat([x, o.view(B, n, HID)], -1).contiguous()
+        rows0 = rows_t.clone() if l in checked else None
+        n_out = cache.select_compact(l, kk, v, rows_t, 2 * HID, n * 2 * HID, 2 * HID, 0)
+        assert n_out == bud["n_out"]
+        kept, posk = cache.kept(l)
+        if l in checked:
+            res = check_kept(kept[0, 0].cpu().numpy(), sc_ref, k, n, L)
+            exact += res == "exact"; ties += res == "tie"
+            idx = kept[0, 0].long()
+            assert torch.equal(rows_t[0, :n_out], rows0[0, idx])
+            assert torch.equal(posk[0, 0], pos[0, idx])
+            Kc, Vc = cache.kv(l)
+            assert torch.equal(Kc[0, 5, :n_out], kk[0, idx, 5]) and torch.equal(Vc[0, 31, :n_out], v[0, idx, 31])
+        xk, ok = rows_t[:, :n_out, :HID].contiguous(), rows_t[:, :n_out, HID:].contiguous()
+        y = pb.glue_linear(ok, W[f"wo{l}"], xk)
+        h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
+        act = pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"]))
+        x = pb.glue_linear(act, W[f"wd{l}"], y)
+        if l in checked:
+            _check_linear(ok, W[f"wo{l}"], y, rng, res=xk)
+            _check_linear(act, W[f"wd{l}"], x, rng, res=y)
+        pos = posk[:, 0].contiguous()
+        del q, kk, v, o, rows_t, h, h2, act, y
+    logits = pb.glue_linear(pb.glue_rmsnorm(x[:, -1].contiguous(), W["nf"]), W["head"])
+    tok = pb.glue_argmax(logits)
+    assert int(tok[0]) == int(synth.widen(logits)[0].argmax())
+    for t in range(T):
+        xt = pb.glue_embed(tok, W["emb"])
+        p = torch.full((B,), N + t, device=DEV, dtype=torch.int32)
+        for l in range(NL):
+            hN = pb.glue_rmsnorm(xt, W[f"n1{l}"])
+            q = pb.glue_rope_(pb.glue_linear(hN, W[f"wq{l}"]).view(B, H, D), p)
+            kn = pb.glue_rope_(pb.glue_linear(hN, W[f"wk{l}"]).view(B, H, D), p)
+            vn = pb.glue_linear(hN, W[f"wv{l}"]).view(B, H, D)
+            o = torch.empty_like(q)
+            if l in checked:
+                Kc, Vc = cache.kv(l)
+                ln = cache.layer_info(l)["len_now"]
+                Kb, Vb = synth.widen(Kc[0, :, :ln]), synth.widen(Vc[0, :, :ln])
+            cache.decode_attn(l, q, kn, vn, o)
+            if l in checked:
+                torch.cuda.synchronize()
+                want, _, _ = oracle.decode_attention(synth.widen(q[0]), Kb, Vb, synth.widen(kn[0]), synth.widen(vn[0]))
+                assert np.abs(synth.widen(o[0]) - want).max() <= 2e-2
+            y = pb.glue_linear(o.view(B, HID), W[f"wo{l}"], xt)
+            h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
+            xt = pb.glue_linear(pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"])), W[f"wd{l}"], y)
+        tok = pb.glue_argmax(pb.glue_linear(pb.glue_rmsnorm(xt, W["nf"]), W["head"]))
+    torch.cuda.synchronize()
+    assert cache.status() == 0
+    assert [cache.layer_info(l)["len_now"] for l in range(NL)] == [b["n_out"] + T for b in budgets]
+    cache.close()
+    print(f"7B-shaped model, batch 1: {exact} of {len(checked)} sampled selections identical to the oracle's, {ties} within the tie band")

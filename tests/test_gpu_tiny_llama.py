@@ -1,8 +1,8 @@
 """The tiny Llama-style workload as a whole model: 2 layers, hidden 256, 4 heads x 64, fp32, batch 2,
 prompt 256, window 32, ratios [1.0, 0.5], 16 greedy decode steps. Attention + score, selection,
-compaction of the hidden rows and decode over the compressed caches run in the CUDA library; the
-decoder glue around them (embedding, RMSNorm, projections, rotary embedding, MLP, output head) is
-plain fp32 torch on the GPU, test harness only. Compared with the fp64 oracle chained through the
+compaction of the hidden rows and decode over the compressed caches run in the CUDA library, and so
+does the decoder glue around them (embedding, RMSNorm, projections, rotary embedding, MLP, output head,
+greedy argmax: the pyr_glue_* kernels); torch only holds the tensors and slices them. Compared with the fp64 oracle chained through the
 same kept sets and tokens (per-call comparison on identical inputs), and with the oracle's own
 free-running generation."""
 import numpy as np
@@ -21,39 +21,38 @@ H, D, HID, L, N, B, STEPS = 4, 64, 256, 32, 256, 2, 16
 
 
 def _rms(x, g, eps=1e-5):
-    return x / torch.sqrt((x * x).mean(-1, keepdim=True) + eps) * g
+    return pb.glue_rmsnorm(x.contiguous(), g, eps)
 
 
 def _rope(x, pos):
-    """x [B, n, H, D] fp32, pos [B, n] ints; the angles are formed in float64."""
-    half = x.shape[-1] // 2
-    theta = 10000.0 ** (-2.0 * torch.arange(half, dtype=torch.float64, device=x.device) / x.shape[-1])
-    ang = pos.to(torch.float64)[..., None, None] * theta
-    cos, sin = torch.cos(ang).float(), torch.sin(ang).float()
-    a, b = x[..., :half], x[..., half:]
-    return torch.cat([a * cos - b * sin, b * cos + a * sin], -1).contiguous()
+    """x [B, n, H, D], pos [B, n] ints -> rotated copy (pyr_glue_rope at the tokens' positions)."""
+    return pb.glue_rope_(x.contiguous().clone(), pos.to(torch.int32).contiguous())
 
 
-def _mlp(x, Wg, Wu, Wd):
-    return (torch.nn.functional.silu(x @ Wg) * (x @ Wu)) @ Wd
+def _lin(x, W, res=None):
+    return pb.glue_linear(x.contiguous(), W, None if res is None else res.contiguous())
+
+
+def _mlp(x, Wg, Wu, Wd, res):
+    return _lin(pb.glue_swiglu(_lin(x, Wg), _lin(x, Wu)), Wd, res)
 
 
 def _gpu_generate(W, ids, ratio, steps):
-    torch.backends.cuda.matmul.allow_tf32 = False
     nL = len(ratio)
+    W = {k: (v.t().contiguous() if v.dim() == 2 and k != "emb" else v) for k, v in W.items()}   # linear weights as [out, in]
     w = dict(n_layers=nL, n_q_heads=H, n_kv_heads=H, head_dim=D, sel_groups=1, dtype="f32", batch=B,
              prompt_len=N, recent_len=L, max_new_tokens=steps)
     cache = pb.PyrCache(device=DEV, **pb.config_from_workload(w, ratio))
-    x = W["emb"][ids]
+    x = pb.glue_embed(ids.to(torch.int32).contiguous(), W["emb"])
     pos = torch.arange(N, device=DEV).expand(B, N).contiguous()
     kepts, scores = [], []
     for l in range(nL):
         n = x.shape[1]
         assert n == cache.layer_info(l)["n_in"]
         h = _rms(x, W[f"n1{l}"])
-        q = _rope((h @ W[f"wq{l}"]).view(B, n, H, D), pos)
-        k = _rope((h @ W[f"wk{l}"]).view(B, n, H, D), pos)
-        v = (h @ W[f"wv{l}"]).view(B, n, H, D).contiguous()
+        q = _rope(_lin(h, W[f"wq{l}"]).view(B, n, H, D), pos)
+        k = _rope(_lin(h, W[f"wk{l}"]).view(B, n, H, D), pos)
+        v = _lin(h, W[f"wv{l}"]).view(B, n, H, D)
         o = torch.empty_like(q)
         cache.prefill_layer(l, q, k, v, o)
         scores.append(cache.scores(l).clone())
@@ -62,26 +61,26 @@ def _gpu_generate(W, ids, ratio, steps):
         n_out = cache.select_compact(l, k, v, rows, 2 * HID, n * 2 * HID, 2 * HID, 0)
         kept, posk = cache.kept(l)
         kepts.append(kept[:, 0].clone())
-        y = rows[:, :n_out, :HID] + rows[:, :n_out, HID:] @ W[f"wo{l}"]
-        x = y + _mlp(_rms(y, W[f"n2{l}"]), W[f"wg{l}"], W[f"wu{l}"], W[f"wd{l}"])
+        y = _lin(rows[:, :n_out, HID:], W[f"wo{l}"], rows[:, :n_out, :HID])
+        x = _mlp(_rms(y, W[f"n2{l}"]), W[f"wg{l}"], W[f"wu{l}"], W[f"wd{l}"], y)
         pos = posk[:, 0].clone().long()
-    logits = [_rms(x[:, -1], W["nf"]) @ W["head"]]
+    logits = [_lin(_rms(x[:, -1], W["nf"]), W["head"])]
     tokens = []
     for t in range(steps):
-        prev = logits[-1].argmax(-1)
-        tokens.append(prev)
-        xt = W["emb"][prev]
+        prev = pb.glue_argmax(logits[-1].contiguous())
+        tokens.append(prev.long())
+        xt = pb.glue_embed(prev, W["emb"])
         p = torch.full((B, 1), N + t, device=DEV)
         for l in range(nL):
             h = _rms(xt, W[f"n1{l}"])
-            q = _rope((h @ W[f"wq{l}"]).view(B, 1, H, D), p)[:, 0].contiguous()
-            k = _rope((h @ W[f"wk{l}"]).view(B, 1, H, D), p)[:, 0].contiguous()
-            v = (h @ W[f"wv{l}"]).view(B, H, D).contiguous()
+            q = _rope(_lin(h, W[f"wq{l}"]).view(B, 1, H, D), p)[:, 0].contiguous()
+            k = _rope(_lin(h, W[f"wk{l}"]).view(B, 1, H, D), p)[:, 0].contiguous()
+            v = _lin(h, W[f"wv{l}"]).view(B, H, D)
             o = torch.empty_like(q)
             cache.decode_attn(l, q, k, v, o)
-            y = xt + o.view(B, HID) @ W[f"wo{l}"]
-            xt = y + _mlp(_rms(y, W[f"n2{l}"]), W[f"wg{l}"], W[f"wu{l}"], W[f"wd{l}"])
-        logits.append(_rms(xt, W["nf"]) @ W["head"])
+            y = _lin(o.view(B, HID), W[f"wo{l}"], xt)
+            xt = _mlp(_rms(y, W[f"n2{l}"]), W[f"wg{l}"], W[f"wu{l}"], W[f"wd{l}"], y)
+        logits.append(_lin(_rms(xt, W["nf"]), W["head"]))
     torch.cuda.synchronize()
     assert cache.status() == 0
     lens = [cache.layer_info(l)["len_now"] for l in range(nL)]

@@ -116,6 +116,10 @@ cudaError_t launch_glue_rmsnorm(const void* x, const void* gain, void* out, int6
                                 cudaStream_t s);
 cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int dtype,
                                cudaStream_t s);
+// bf16 tensor-core GEMM of the glue (csrc/gemm_tc.cu): y = x w^T (+ res); w is [N, K]
+bool gemm_tc_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
+cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
+                           cudaStream_t s);
 cudaError_t launch_glue_rope(void* x, const int32_t* pos, int64_t tokens, int H, int D, int dtype, cudaStream_t s);
 cudaError_t launch_glue_swiglu(const void* g, const void* u, void* out, int64_t n, int dtype, cudaStream_t s);
 cudaError_t launch_glue_argmax(const void* x, int32_t* out, int64_t rows, int n, int dtype, cudaStream_t s);

@@ -45,3 +45,30 @@ def test_glue_kernels_against_fp64(dtype, tol):
     am = pb.glue_argmax(lg).cpu().numpy()
     assert am[2] == 17 and am[4] == 0
     np.testing.assert_array_equal(am[[0, 1, 3, 5]], synth.widen(lg).argmax(-1)[[0, 1, 3, 5]])
+
+
+@pytest.mark.parametrize("M,N,K,res", [(300, 512, 256, False), (64, 4096, 4096, True), (2048, 11008, 4096, True),
+                                       (129, 1000, 64, False), (5000, 4096, 11008, False), (1, 32000, 4096, False)])
+def test_tensor_core_linear_against_fp64_samples(M, N, K, res):
+    """bf16 pyr_glue_linear with K a multiple of 64 runs on the tcgen05 GEMM: sampled entries (first and
+    last rows and columns among them) against fp64 dot products of the bf16 inputs, untouched padding."""
+    x = _r(M, K, seed=21, dtype=torch.bfloat16)
+    w = (_r(N, K, seed=22) * 0.05).to(torch.bfloat16)
+    r = _r(M, N, seed=23, dtype=torch.bfloat16) if res else None
+    launches = pb.launch_count()
+    y = pb.glue_linear(x, w, r)
+    torch.cuda.synchronize()
+    assert pb.launch_count() - launches == 1
+    rng = np.random.default_rng(M + N)
+    rows = np.concatenate([[0, M - 1, min(127, M - 1), min(128, M - 1)], rng.integers(0, M, size=60)])
+    cols = np.concatenate([[0, N - 1, min(255, N - 1), min(256, N - 1)], rng.integers(0, N, size=60)])
+    rt, ct = torch.from_numpy(rows).to(DEV), torch.from_numpy(cols).to(DEV)
+    want = (x[rt].double() * w[ct].double()).sum(-1)
+    if res:
+        want = want + r[rt, ct].double()
+    got = y[rt, ct].double()
+    scale = float(want.abs().max().clamp_min(1e-3))
+    assert float((got - want).abs().max()) <= 2 ** -7 * scale
+    # a whole row and a whole column
+    np.testing.assert_allclose(synth.widen(y[M // 2]), synth.widen(x[M // 2]) @ synth.widen(w).T + (synth.widen(r[M // 2]) if res else 0),
+                               atol=2 ** -7 * scale, rtol=2 ** -7)

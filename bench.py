@@ -247,6 +247,176 @@ class Workload:
         return tot
 
 
+class ModelWorkload(Workload):
+    """The 7B-shaped workload as a whole model on the library's kernels: embedding, RMSNorm, the
+    projections and the MLP on the tcgen05 GEMM, rotary embedding at original positions, the pyramid
+    path, o_proj on all rows followed by the in-place compaction of the hidden rows, greedy head.
+    torch holds the tensors (and makes the compacted rows contiguous between layers)."""
+
+    def __init__(self, name: str, device, layers: int = 0, decode_steps: int = -1, batch: int = 0, reselect_every: int = 0):
+        from paper_2405_12532_b200 import binding as pb
+        self.pb = pb
+        self.name = name
+        self.w = w = dict(synth.CONFIGS[name])
+        self.device = device
+        self.ratio = synth.ratio_schedule(w)
+        if layers > 0:
+            self.ratio = self.ratio[:layers]
+            w["n_layers"] = layers
+        if decode_steps >= 0:
+            w["max_new_tokens"] = decode_steps
+        if batch > 0:
+            w["batch"] = batch
+        self.reselect_every = reselect_every
+        flags = pb.PYR_FLAG_GEN_RESELECT if reselect_every else 0
+        self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio, flags=flags))
+        self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
+        self.dt = torch.bfloat16
+        self.eb = 2
+        self.G = 1
+        self.T = w["max_new_tokens"]
+        B, N, d, f, V = w["batch"], w["prompt_len"], w["hidden"], w["inter"], w["vocab"]
+        g = torch.Generator(device=device)
+        g.manual_seed(1)
+        rn = lambda *s: (torch.randn(*s, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        self.W = {"emb": rn(V, d), "head": rn(V, d), "nf": torch.ones(d, device=device, dtype=torch.bfloat16)}
+        for l in range(w["n_layers"]):
+            for nm, shape in (("wq", (d, d)), ("wk", (d, d)), ("wv", (d, d)), ("wo", (d, d)), ("wg", (f, d)), ("wu", (f, d)), ("wd", (d, f))):
+                self.W[f"{nm}{l}"] = rn(*shape)
+            self.W[f"n1{l}"] = torch.ones(d, device=device, dtype=torch.bfloat16)
+            self.W[f"n2{l}"] = torch.ones(d, device=device, dtype=torch.bfloat16)
+        self.ids = synth.uniform_token_ids(B, N, V, seed=0).to(torch.int32).to(device)
+        self.dec_ids = synth.uniform_token_ids(B, max(self.T, 1), V, seed=2).to(torch.int32).to(device)
+        self.out = None
+        self.rows = None
+
+    def prefill(self, events=None):
+        pb, W, w = self.pb, self.W, self.w
+        B, N, H, D, d = w["batch"], w["prompt_len"], w["n_q_heads"], w["head_dim"], w["hidden"]
+        c = self.cache
+        c.reset()
+        x = pb.glue_embed(self.ids, W["emb"])
+        pos = torch.arange(N, device=self.device, dtype=torch.int32).expand(B, N).contiguous()
+        for l in range(w["n_layers"]):
+            n = x.shape[1]
+            if events is not None:
+                events[l][0].record()
+            h = pb.glue_rmsnorm(x, W[f"n1{l}"])
+            q = pb.glue_rope_(pb.glue_linear(h, W[f"wq{l}"]).view(B, n, H, D), pos)
+            k = pb.glue_rope_(pb.glue_linear(h, W[f"wk{l}"]).view(B, n, H, D), pos)
+            v = pb.glue_linear(h, W[f"wv{l}"]).view(B, n, H, D)
+            o = torch.empty_like(q)
+            c.prefill_layer(l, q, k, v, o)
+            y = pb.glue_linear(o.view(B, n, d), W[f"wo{l}"], x)
+            if events is not None:
+                events[l][1].record()
+            n_out = c.select_compact(l, k, v, y, d, n * d, d, 0)
+            if events is not None:
+                events[l][2].record()
+            y = y[:, :n_out].contiguous()
+            pos = c.kept(l)[1][:, 0].contiguous()
+            h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
+            x = pb.glue_linear(pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"])), W[f"wd{l}"], y)
+        logits = pb.glue_linear(pb.glue_rmsnorm(x[:, -1].contiguous(), W["nf"]), W["head"])
+        self.first_token = pb.glue_argmax(logits)
+
+    def decode(self):
+        pb, W, w = self.pb, self.W, self.w
+        B, N, H, D, d = w["batch"], w["prompt_len"], w["n_q_heads"], w["head_dim"], w["hidden"]
+        c = self.cache
+        for t in range(self.T):
+            xt = pb.glue_embed(self.dec_ids[:, t].contiguous(), W["emb"])      # pre-drawn ids: the timing does not hang on ties
+            p = torch.full((B,), N + t, device=self.device, dtype=torch.int32)
+            for l in range(w["n_layers"]):
+                h = pb.glue_rmsnorm(xt, W[f"n1{l}"])
+                q = pb.glue_rope_(pb.glue_linear(h, W[f"wq{l}"]).view(B, H, D), p)
+                k = pb.glue_rope_(pb.glue_linear(h, W[f"wk{l}"]).view(B, H, D), p)
+                v = pb.glue_linear(h, W[f"wv{l}"]).view(B, H, D)
+                o = torch.empty_like(q)
+                c.decode_attn(l, q, k, v, o)
+                y = pb.glue_linear(o.view(B, d), W[f"wo{l}"], xt)
+                h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
+                xt = pb.glue_linear(pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"])), W[f"wd{l}"], y)
+            self.last_token = pb.glue_argmax(pb.glue_linear(pb.glue_rmsnorm(xt, W["nf"]), W["head"]))
+            if self.reselect_every and (t + 1) % self.reselect_every == 0:
+                for l in range(w["n_layers"]):
+                    c.decode_reselect(l)
+
+    def linear_flops(self):
+        w = self.w
+        B, d, f = w["batch"], w["hidden"], w["inter"]
+        tot = 0
+        for L in self.layers:
+            n_out = L["k_ctx"] + min(w["recent_len"], L["n_in"])
+            tot += 2 * B * L["n_in"] * 4 * d * d + 2 * B * n_out * 3 * d * f
+        return tot + 2 * B * d * w["vocab"]
+
+    def weight_bytes(self):
+        w = self.w
+        d, f = w["hidden"], w["inter"]
+        return (w["n_layers"] * (4 * d * d + 3 * d * f) + d * w["vocab"]) * 2
+
+    def select_args(self, l, n):
+        raise NotImplementedError
+
+
+def run_model(args, rank, world, local_rank, name):
+    """One line for the whole-model workload: the same step (prefill of all layers, then T decode steps),
+    now with the model's linear layers, norms, rotary embedding and head inside it."""
+    from paper_2405_12532_b200 import binding as pb
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    wl = ModelWorkload(name, device, layers=args.layers, decode_steps=args.decode_steps, batch=args.batch,
+                       reselect_every=args.reselect_every)
+    w = wl.w
+    hbm, tf_burst, tf_sust, peak_src = measured_peaks()
+    for _ in range(args.warmup):
+        wl.prefill(); wl.decode()
+    pdist.barrier(world)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = pb.launch_count()
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    pdist.barrier(world)
+    for s in range(args.steps):
+        marks[s][0].record(); wl.prefill(); marks[s][1].record(); wl.decode(); marks[s][2].record()
+    pdist.barrier(world)
+    launches = pb.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    assert wl.cache.status() == 0
+    t_pre = sum(m[0].elapsed_time(m[1]) for m in marks) / 1e3
+    t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
+    t_pre, t_dec = pdist.max_over_ranks([t_pre, t_dec], world, device)
+    if rank != 0:
+        return
+    K, B, N, T = args.steps, w["batch"], w["prompt_len"], w["max_new_tokens"]
+    flops = wl.linear_flops() + wl.prefill_flops()
+    dec_bytes = wl.decode_bytes() + T * wl.weight_bytes()
+    ach = K * flops / t_pre / 1e12
+    line = {"metric": METRIC, "value": world * K * B * N / t_pre,
+            "unit": "tokens/s (prefill, whole model: linear layers, norms, rotary embedding and the attention path)",
+            "decode_tokens_per_s": world * K * B * T / t_dec if T > 0 else None,
+            "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": (t_pre + t_dec) / K * 1e3,
+            "ms_prefill": t_pre / K * 1e3, "ms_decode": t_dec / K * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "scope": "whole model on the library's kernels; random-init weights, uniform random token ids",
+                       "layers": w["n_layers"], "batch_per_gpu": B, "prompt_len": N, "recent_len": w["recent_len"],
+                       "decode_steps": T, "hidden": w["hidden"], "inter": w["inter"], "vocab": w["vocab"],
+                       "ratio": "geometric 1.0->%.2f" % wl.ratio[-1], "reselect_every": args.reselect_every or None,
+                       "l2": "weights (13.5 GB) and activations are far larger than L2"},
+            "roofline": {"kernel": "prefill: linear layers (tcgen05 GEMM) + attention path", "bound": "tensor", "achieved": ach,
+                         "peak": tf_burst, "unit": "TFLOP/s", "frac": ach / tf_burst, "frac_of_sustained": ach / tf_sust,
+                         "traffic": None, "peak_source": f"of {peak_src}"},
+            "roofline_decode": ({"kernel": "decode: weights streamed once per step + K/V caches", "bound": "hbm",
+                                 "achieved": K * dec_bytes / t_dec / 1e9, "peak": hbm, "unit": "GB/s",
+                                 "frac": K * dec_bytes / t_dec / 1e9 / hbm, "traffic": None, "peak_source": f"of {peak_src}"}
+                                if T > 0 else None),
+            "gpu_launches": launches, "clocks": clocks, "e2e": None, "cpu_baseline": None}
+    print(json.dumps(line), flush=True)
+    wl.cache.close()
+
+
 def run_ours(args, rank, world, local_rank, workload=None):
     from paper_2405_12532_b200 import binding as pb
     name = workload or args.workload
@@ -530,7 +700,10 @@ def run(args):
     try:
         names = list(synth.CONFIGS) if args.workload == "all" else [args.workload]
         for name in names:          # "all": one line per workload, back to back
-            run_ours(args, rank, world, local_rank, name)
+            if synth.CONFIGS[name]["kind"] == "model":
+                run_model(args, rank, world, local_rank, name)
+            else:
+                run_ours(args, rank, world, local_rank, name)
             torch.cuda.empty_cache()
     finally:
         if world > 1:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpyr.so")
-SOURCES = ["pyr_host.cu", "prefill_simt.cu", "prefill_tc.cu", "attn_tc.cu", "select_compact.cu", "decode.cu", "decode_noalloc.cu", "gen_reselect.cu", "glue.cu", "gemm_tc.cu"]
+SOURCES = ["pyr_host.cu", "prefill_simt.cu", "prefill_tc.cu", "attn_tc.cu", "select_compact.cu", "decode.cu", "decode_noalloc.cu", "gen_reselect.cu", "glue.cu", "gemm_tc.cu", "gemm_skinny.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -509,6 +509,8 @@ pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual,
   if (!glue_ok(dtype, {x, w, y})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
   if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
   if (m == 0) return PYR_OK;
+  if (dtype == PYR_BF16 && pyr::gemm_skinny_supported(x, w, residual, y, m, n, k))
+    PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
   if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
     PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
   PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, static_cast<cudaStream_t>(stream)));

@@ -43,6 +43,13 @@ CONFIGS = {
                             dtype="bf16", batch=8, prompt_len=256, recent_len=102,
                             ratio=(1.0, 0.2), sel_groups=8, max_new_tokens=128,
                             hitter_frac=0.01, hitter_mag=4.0),
+    # The 7B workload as a whole model: the same attention geometry, window and schedule as 7b_64x2k with
+    # the public Llama-2-7B block around it (hidden 4096, MLP 11008, vocabulary 32000), random-init weights,
+    # uniform random token ids for the prompt and for the decode steps.
+    "7b_model_64x2k": dict(kind="model", n_layers=32, n_q_heads=32, n_kv_heads=32, head_dim=128,
+                           dtype="bf16", batch=64, prompt_len=2048, recent_len=256,
+                           ratio=(1.0, 0.3), sel_groups=1, max_new_tokens=128,
+                           hitter_frac=0.0, hitter_mag=0.0, hidden=4096, inter=11008, vocab=32000),
 }
 
 

@@ -72,3 +72,22 @@ def test_tensor_core_linear_against_fp64_samples(M, N, K, res):
     # a whole row and a whole column
     np.testing.assert_allclose(synth.widen(y[M // 2]), synth.widen(x[M // 2]) @ synth.widen(w).T + (synth.widen(r[M // 2]) if res else 0),
                                atol=2 ** -7 * scale, rtol=2 ** -7)
+
+
+@pytest.mark.parametrize("M,N,K,res", [(64, 4096, 11008, True), (37, 11008, 4096, False), (17, 128, 64, False),
+                                       (64, 64, 512, True), (1, 4096, 4096, True), (65, 4096, 4096, True)])
+def test_skinny_linear_whole_output(M, N, K, res):
+    """At most 64 rows: the weight-streaming kernel (K slices summed across a cluster in slice order).
+    The whole output against fp64, and bit-identical on a second run; 65 rows take the tcgen05 path."""
+    x = _r(M, K, seed=31, dtype=torch.bfloat16)
+    w = (_r(N, K, seed=32) * 0.05).to(torch.bfloat16)
+    r = _r(M, N, seed=33, dtype=torch.bfloat16) if res else None
+    y = pb.glue_linear(x, w, r)
+    y2 = pb.glue_linear(x, w, r)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+    want = x.double() @ w.double().T
+    if res:
+        want = want + r.double()
+    scale = float(want.abs().max().clamp_min(1e-3))
+    assert float((y.double() - want).abs().max()) <= 2 ** -7 * scale

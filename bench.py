@@ -35,6 +35,7 @@ UNIT = "tokens/s (prefill of the attention path, all layers incl. select+compact
 SCOPE = ("attention path only: per-layer Q/K/V are inputs; a full model's projections, MLP and weight reads "
          "are not in the step")
 DEFAULT_WORKLOAD = "7b_64x2k"
+MODEL_WORKLOAD = "7b_model_64x2k"      # the same shapes as a whole model; reported beside the default line
 PROFILES = os.path.join(ROOT, "profiles")
 
 
@@ -159,6 +160,13 @@ class Workload:
         self.T = w["max_new_tokens"]
         self.dec_in = [synth.decode_step_inputs(w, 0, t, device=device) for t in range(4)]
         self.dec_out = torch.empty(B, Hq, D, dtype=self.dt, device=device)
+
+    def release(self):
+        """Give the device memory back (the schedule-derived accounting below stays usable)."""
+        if self.cache is not None:
+            self.cache.close()
+        self.cache = self.pool = self.out = self.rows = self.dec_in = self.dec_out = None
+        torch.cuda.empty_cache()
 
     def layer_views(self, l):
         n = self.layers[l]["n_in"]
@@ -360,9 +368,10 @@ class ModelWorkload(Workload):
         raise NotImplementedError
 
 
-def run_model(args, rank, world, local_rank, name):
+def run_model(args, rank, world, local_rank, name, emit=True):
     """One line for the whole-model workload: the same step (prefill of all layers, then T decode steps),
-    now with the model's linear layers, norms, rotary embedding and head inside it."""
+    now with the model's linear layers, norms, rotary embedding and head inside it. With emit=False the
+    line is returned (rank 0; None elsewhere) instead of printed."""
     from paper_2405_12532_b200 import binding as pb
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
@@ -388,8 +397,11 @@ def run_model(args, rank, world, local_rank, name):
     t_pre = sum(m[0].elapsed_time(m[1]) for m in marks) / 1e3
     t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
     t_pre, t_dec = pdist.max_over_ranks([t_pre, t_dec], world, device)
+    wl.cache.close()
+    wl.cache = wl.W = None
+    torch.cuda.empty_cache()
     if rank != 0:
-        return
+        return None
     K, B, N, T = args.steps, w["batch"], w["prompt_len"], w["max_new_tokens"]
     flops = wl.linear_flops() + wl.prefill_flops()
     dec_bytes = wl.decode_bytes() + T * wl.weight_bytes()
@@ -413,8 +425,9 @@ def run_model(args, rank, world, local_rank, name):
                                  "frac": K * dec_bytes / t_dec / 1e9 / hbm, "traffic": None, "peak_source": f"of {peak_src}"}
                                 if T > 0 else None),
             "gpu_launches": launches, "clocks": clocks, "e2e": None, "cpu_baseline": None}
-    print(json.dumps(line), flush=True)
-    wl.cache.close()
+    if emit:
+        print(json.dumps(line), flush=True)
+    return line
 
 
 def run_ours(args, rank, world, local_rank, workload=None):
@@ -467,6 +480,13 @@ def run_ours(args, rank, world, local_rank, workload=None):
 
     # ---- end to end: host buffers, copies inside the timed region
     e2e = run_e2e(wl, args, barrier, world) if not args.no_e2e else None
+    wl.release()
+
+    # the same 7B shapes as a whole model (linear layers, norms, rotary embedding, head), reported beside the
+    # attention-path numbers of the headline line
+    model = None
+    if name == DEFAULT_WORKLOAD and not args.no_model and not (args.layers or args.batch or args.decode_steps >= 0):
+        model = run_model(args, rank, world, local_rank, MODEL_WORKLOAD, emit=False)
 
     if rank != 0:
         return
@@ -523,8 +543,11 @@ def run_ours(args, rank, world, local_rank, workload=None):
         "gpu_launches": launches, "wall_s": wall, "clocks": clocks, "e2e": e2e,
         "cpu_baseline": cpu_baseline(name) if not args.no_cpu else None,
     }
+    if model is not None:
+        line["whole_model"] = {k: model[k] for k in ("value", "unit", "decode_tokens_per_s", "ms_prefill", "ms_decode",
+                                                      "roofline", "roofline_decode", "gpu_launches", "clocks")}
+        line["whole_model"]["workload"] = MODEL_WORKLOAD
     print(json.dumps(line), flush=True)
-    wl.cache.close()
 
 
 def run_e2e(wl, args, barrier, world):
@@ -699,6 +722,8 @@ def run(args):
         pdist.init("nccl", torch.device("cuda", local_rank))
     try:
         names = list(synth.CONFIGS) if args.workload == "all" else [args.workload]
+        if args.workload == "all":
+            args.no_model = True    # the whole-model workload has its own line in this mode
         for name in names:          # "all": one line per workload, back to back
             if synth.CONFIGS[name]["kind"] == "model":
                 run_model(args, rank, world, local_rank, name)
@@ -726,6 +751,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-model", action="store_true", help="skip the whole-model run that the default workload reports beside its line")
     ap.add_argument("--reselect-every", type=int, default=0,
                     help="generation-phase PvC update of every layer every so many decode steps (0: never)")
     ap.add_argument("--dry-run", action="store_true", help="launch path only (gloo, no GPU work)")

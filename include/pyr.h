@@ -312,14 +312,18 @@ pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
 /*
  * Decoder glue for whole-model workloads. (No counterpart in the paper beyond Appendix A.2's
  * choice of positions: these are the public Llama block's steps around the pyramid path, so that a
- * model can run end to end on this library's kernels. CUDA-core kernels, fp32 arithmetic, for fp32
- * or bf16 storage; dtype is a pyr_dtype_t.) All pointers are device pointers, tensors row-major and
- * contiguous, every call asynchronous on `stream`.
+ * model can run end to end on this library's kernels. fp32 arithmetic for fp32 or bf16 storage;
+ * dtype is a pyr_dtype_t. CUDA-core kernels, except the bf16 linear layer, see below.) All pointers
+ * are device pointers, tensors row-major and contiguous, every call asynchronous on `stream`.
  *   embed   out[t, :] = table[ids[t], :]; table [vocab, d]. An id outside [0, vocab) zeroes its row
  *           and, if dev_status (a device int, may be NULL) is given, records PYR_ERR_INVALID in it.
  *   rmsnorm out = x / sqrt(mean(x^2) + eps) * gain; x, out [tokens, d] (may alias), gain [d].
  *   linear  y[m, n] = x[m, k] . w[n, k] (+ residual[m, n] if not NULL); w is [n, k] ("out, in").
- *           y may alias residual, not x.
+ *           y may alias residual, not x. bf16 with 16-byte aligned pointers and k a multiple of 64
+ *           runs on tensor cores (fp32 accumulation, one rounding to bf16 at the end): for m <= 64
+ *           and n a multiple of 128 a weight-streaming kernel whose clusters split k and add their
+ *           partial sums in a fixed order, else a tiled kernel (n a multiple of 8). Results are
+ *           bit-reproducible run to run in every case. Everything else takes the CUDA-core kernel.
  *   rope    rotates, in place, the pairs (i, i + head_dim/2) of every head of x [tokens, n_heads,
  *           head_dim] by pos[t] * 10000^(-2i/head_dim): Appendix A.2's "gather" when pos holds the
  *           tokens' original positions (pyr_cache_kept's second pointer), "re-encode" when it counts

@@ -324,7 +324,7 @@ class ModelWorkload(Workload):
             y = y[:, :n_out].contiguous()
             pos = c.kept(l)[1][:, 0].contiguous()
             h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
-            x = pb.glue_linear(pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"])), W[f"wd{l}"], y)
+            x = pb.glue_linear(pb.glue_linear_swiglu(h2, W[f"wg{l}"], W[f"wu{l}"]), W[f"wd{l}"], y)
         logits = pb.glue_linear(pb.glue_rmsnorm(x[:, -1].contiguous(), W["nf"]), W["head"])
         self.first_token = pb.glue_argmax(logits)
 

@@ -324,10 +324,14 @@ pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
  *           and n a multiple of 128 a weight-streaming kernel whose clusters split k and add their
  *           partial sums in a fixed order, else a tiled kernel (n a multiple of 8). Results are
  *           bit-reproducible run to run in every case. Everything else takes the CUDA-core kernel.
+ *   linear_swiglu  out[m, n] = silu(x . w_gate^T) * (x . w_up^T), w_gate and w_up [n, k]: the gated MLP's
+ *           first half in one pass, neither projection written out (fp32 accumulators go straight
+ *           into the product). bf16 with 16-byte aligned pointers, k a multiple of 64 and n a
+ *           multiple of 8 only; PYR_ERR_UNSUPPORTED otherwise (call linear twice and swiglu).
  *   rope    rotates, in place, the pairs (i, i + head_dim/2) of every head of x [tokens, n_heads,
  *           head_dim] by pos[t] * 10000^(-2i/head_dim): Appendix A.2's "gather" when pos holds the
  *           tokens' original positions (pyr_cache_kept's second pointer), "re-encode" when it counts
- *           from 0.
+ *           from 0. head_dim at most 256.
  *   swiglu  out = silu(gate) * up, n elements.
  *   argmax  out[r] = index of the largest of x[r, 0..n), the lowest index on ties; x [rows, n].
  */
@@ -337,6 +341,8 @@ pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_
                               int32_t dtype, void* stream);
 pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual, void* y, int64_t m, int32_t n,
                              int32_t k, int32_t dtype, void* stream);
+pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
+                                    int32_t k, int32_t dtype, void* stream);
 pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,
                            int32_t dtype, void* stream);
 pyr_status_t pyr_glue_swiglu(const void* gate, const void* up, void* out, int64_t n, int32_t dtype, void* stream);

@@ -25,7 +25,7 @@ PYR_FLAG_POS_REENCODE = 4
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_swiglu",
     "pyr_glue_rope", "pyr_glue_swiglu", "pyr_glue_argmax", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         L.pyr_glue_embed.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp, vp]
         L.pyr_glue_rmsnorm.argtypes = [vp, vp, vp, i64, i32, C.c_float, i32, vp]
         L.pyr_glue_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
+        L.pyr_glue_linear_swiglu.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
         L.pyr_glue_rope.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.pyr_glue_swiglu.argtypes = [vp, vp, vp, i64, i32, vp]
         L.pyr_glue_argmax.argtypes = [vp, vp, i64, i32, i32, vp]
@@ -195,6 +196,16 @@ def glue_linear(x, w, residual=None):
     _check(lib().pyr_glue_linear(x.data_ptr(), w.data_ptr(), residual.data_ptr() if residual is not None else None,
                                  y.data_ptr(), x.numel() // K, N, K, _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_linear")
     return y
+
+
+def glue_linear_swiglu(x, w_gate, w_up):
+    """silu(x . w_gate^T) * (x . w_up^T) -> [..., N] in one pass (pyr_glue_linear_swiglu; bf16, K a multiple of 64)."""
+    assert x.is_contiguous() and w_gate.is_contiguous() and w_up.is_contiguous() and w_gate.shape == w_up.shape
+    N, K = w_gate.shape
+    out = torch.empty(*x.shape[:-1], N, dtype=x.dtype, device=x.device)
+    _check(lib().pyr_glue_linear_swiglu(x.data_ptr(), w_gate.data_ptr(), w_up.data_ptr(), out.data_ptr(), x.numel() // K, N, K,
+                                        _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_linear_swiglu")
+    return out
 
 
 def glue_rope_(x, pos):

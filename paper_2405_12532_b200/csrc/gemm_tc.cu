@@ -10,6 +10,11 @@
 // Two accumulator buffers of BN columns: the epilogue of a tile overlaps the main loop of the next.
 // Tiles are ordered so that the CTAs running at one time share a band of 16 row blocks of x and a
 // few column blocks of w, which stay in L2. Every barrier is followed phase by phase by its waiter.
+//
+// The gated form (kGated) computes out = silu(x . wg^T) * (x . wu^T) in one pass: a 256-column tile is
+// 128 rows of wg beside the same 128 rows of wu (two TMA boxes into one stage), the accumulator holds
+// the gate in columns 0-127 and the up projection in 128-255, and the epilogue multiplies them, so
+// neither projection is ever written out.
 #include <cuda_bf16.h>
 #include <stddef.h>
 
@@ -58,15 +63,18 @@ __device__ __forceinline__ void tile_of(int tile, int mblocks, int nblocks, int*
   *mb = m0 + in % rows;
 }
 
-template <int BN>
+template <int BN, bool kGated>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, GemmArgs a) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+               const __grid_constant__ CUtensorMap map_w2, GemmArgs a) {
+  static_assert(!kGated || BN == 256, "the gated form pairs two 128-row boxes");
+  constexpr int kOutCols = kGated ? BN / 2 : BN;       // output columns per tile
   using Cfg = GemmCfg<BN>;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   GemmSmem<BN>& sm = *reinterpret_cast<GemmSmem<BN>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mblocks = (int)((a.M + kBM - 1) / kBM), nblocks = (a.N + BN - 1) / BN;
+  const int mblocks = (int)((a.M + kBM - 1) / kBM), nblocks = (a.N + kOutCols - 1) / kOutCols;
   const int tiles = mblocks * nblocks;
   const int ksteps = a.K / kBK;
   volatile int* abort_flag = &sm.abort_flag;
@@ -92,6 +100,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (lane == 0) {
       prefetch_tensormap(&map_x);
       prefetch_tensormap(&map_w);
+      if (kGated) prefetch_tensormap(&map_w2);
       bool ok = true;
       int it = 0;                                 // stages filled so far
       for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
@@ -103,7 +112,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           if (!ok) break;
           mbar_expect_tx(&sm.full[st], Cfg::kABytes + Cfg::kBBytes);
           tma_load_4d(sm.a[st], &map_x, &sm.full[st], ks * kBK, 0, mb * kBM, 0);
-          tma_load_4d(sm.b[st], &map_w, &sm.full[st], ks * kBK, 0, nb * BN, 0);
+          if (kGated) {
+            tma_load_4d(sm.b[st], &map_w, &sm.full[st], ks * kBK, 0, nb * kOutCols, 0);
+            tma_load_4d(sm.b[st] + Cfg::kBBytes / 2, &map_w2, &sm.full[st], ks * kBK, 0, nb * kOutCols, 0);
+          } else {
+            tma_load_4d(sm.b[st], &map_w, &sm.full[st], ks * kBK, 0, nb * BN, 0);
+          }
         }
       }
     }
@@ -150,13 +164,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       const int64_t m = (int64_t)mb * kBM + row;
-      const int n0 = nb * BN;
+      const int n0 = nb * kOutCols;
 #pragma unroll 1
-      for (int c32 = 0; c32 < BN / 32; ++c32) {
+      for (int c32 = 0; c32 < kOutCols / 32; ++c32) {
         uint32_t v[32];
         tmem_ld32(t_base + buf * BN + c32 * 32, v);
-        tmem_wait_ld();
-        if (c32 == BN / 32 - 1) {                 // the buffer is in registers: the tile after next may use it
+        if (kGated) {
+          uint32_t u[32];
+          tmem_ld32(t_base + buf * BN + kOutCols + c32 * 32, u);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float g = __uint_as_float(v[e]);
+            v[e] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(u[e]));
+          }
+        } else {
+          tmem_wait_ld();
+        }
+        if (c32 == kOutCols / 32 - 1) {           // the buffer is in registers: the tile after next may use it
           tc_fence_before();
           mbar_arrive(&sm.acc_empty[buf]);
         }
@@ -196,14 +221,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   }
 }
 
-template <int BN>
-cudaError_t run_gemm(const CUtensorMap& mx, const CUtensorMap& mw, const GemmArgs& a, int sms, cudaStream_t s) {
+template <int BN, bool kGated>
+cudaError_t run_gemm(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& mw2, const GemmArgs& a, int sms,
+                     cudaStream_t s) {
   const size_t smem = sizeof(GemmSmem<BN>) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, kGated>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const long long tiles = ((a.M + kBM - 1) / kBM) * (long long)((a.N + BN - 1) / BN);
+  const int out_cols = kGated ? BN / 2 : BN;
+  const long long tiles = ((a.M + kBM - 1) / kBM) * (long long)((a.N + out_cols - 1) / out_cols);
   const int grid = (int)(tiles < sms ? tiles : sms);
-  gemm_tc_kernel<BN><<<grid, kGemmThreads, smem, s>>>(mx, mw, a);
+  gemm_tc_kernel<BN, kGated><<<grid, kGemmThreads, smem, s>>>(mx, mw, mw2, a);
   return cudaGetLastError();
 }
 
@@ -229,7 +256,23 @@ cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* 
   GemmArgs a;
   a.res = static_cast<const __nv_bfloat16*>(res); a.y = static_cast<__nv_bfloat16*>(y);
   a.M = M; a.N = N; a.K = K; a.status = status;
-  return BN == 256 ? run_gemm<256>(mx, mw, a, sms, s) : run_gemm<128>(mx, mw, a, sms, s);
+  return BN == 256 ? run_gemm<256, false>(mx, mw, mw, a, sms, s) : run_gemm<128, false>(mx, mw, mw, a, sms, s);
+}
+
+// out[M, N] = silu(x . wg^T) * (x . wu^T): the gated form of the kernel above
+cudaError_t launch_gemm_tc_gated(const void* x, const void* wg, const void* wu, void* out, int64_t M, int N, int K,
+                                 int* status, cudaStream_t s) {
+  const int sms = device_sm_count();
+  if (sms <= 0) return cudaErrorUnknown;
+  CUtensorMap mx, mg, mu;
+  if (!make_tensor_map_bf16(&mx, x, 1, (int)M, 1, K, (int64_t)M * K, K, K, kBM) ||
+      !make_tensor_map_bf16(&mg, wg, 1, N, 1, K, (int64_t)N * K, K, K, 128) ||
+      !make_tensor_map_bf16(&mu, wu, 1, N, 1, K, (int64_t)N * K, K, K, 128))
+    return cudaErrorInvalidValue;
+  GemmArgs a;
+  a.res = nullptr; a.y = static_cast<__nv_bfloat16*>(out);
+  a.M = M; a.N = N; a.K = K; a.status = status;
+  return run_gemm<256, true>(mx, mg, mu, a, sms, s);
 }
 
 }  // namespace pyr

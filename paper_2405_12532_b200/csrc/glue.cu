@@ -84,22 +84,31 @@ __global__ void __launch_bounds__(256) linear_kernel(const T* x, const T* w, con
     }
 }
 
-// rotate the pairs (i, i + D/2) of every head of token t by pos[t] * 10000^(-2i/D); the angle in double
+// rotate the pairs (i, i + D/2) of every head of token t by pos[t] * 10000^(-2i/D). One CTA per token:
+// the D/2 angles are the same for all heads, so they are taken once (in double: positions reach the
+// thousands and the fp32 model is held to 1e-4) and kept in shared memory as fp32 cosines and sines.
+constexpr int kRopeMaxHalf = 128;
 template <typename T>
-__global__ void rope_kernel(T* x, const int32_t* pos, int64_t tokens, int H, int D) {
+__global__ void __launch_bounds__(256) rope_kernel(T* x, const int32_t* pos, int64_t tokens, int H, int D) {
+  __shared__ float2 cs[kRopeMaxHalf];
   const int half = D / 2;
-  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= tokens * H * half) return;
-  const int i = (int)(e % half);
-  const int64_t th = e / half;                 // token * H + head
-  const int64_t t = th / H;
-  const double ang = (double)pos[t] * exp2(-2.0 * (double)i / (double)D * 13.287712379549449);   // log2(10000)
-  double sn, cs;
-  sincos(ang, &sn, &cs);
-  T* p = x + th * D;
-  const float a = ld(p + i), b = ld(p + i + half);
-  st(p + i, (float)((double)a * cs - (double)b * sn));
-  st(p + i + half, (float)((double)b * cs + (double)a * sn));
+  const int64_t t = blockIdx.x;
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    const double ang = (double)pos[t] * exp2(-2.0 * (double)i / (double)D * 13.287712379549449);   // log2(10000)
+    double sn, c;
+    sincos(ang, &sn, &c);
+    cs[i] = make_float2((float)c, (float)sn);
+  }
+  __syncthreads();
+  T* row = x + t * (int64_t)H * D;
+  for (int e = threadIdx.x; e < H * half; e += blockDim.x) {
+    const int i = e % half, h = e / half;
+    T* p = row + h * D;
+    const float a = ld(p + i), b = ld(p + i + half);
+    const float2 w = cs[i];
+    st(p + i, a * w.x - b * w.y);
+    st(p + i + half, b * w.x + a * w.y);
+  }
 }
 
 template <typename T>
@@ -166,9 +175,9 @@ cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, vo
       [&] { linear_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, (const __nv_bfloat16*)res, (__nv_bfloat16*)y, M, N, K); });
 }
 cudaError_t launch_glue_rope(void* x, const int32_t* pos, int64_t tokens, int H, int D, int dtype, cudaStream_t s) {
-  const int64_t n = tokens * H * (D / 2);
-  if (n == 0) return cudaSuccess;
-  const unsigned blocks = (unsigned)((n + 255) / 256);
+  if (tokens == 0) return cudaSuccess;
+  if (D / 2 > kRopeMaxHalf || tokens > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const unsigned blocks = (unsigned)tokens;
   return by_dtype(dtype,
       [&] { rope_kernel<float><<<blocks, 256, 0, s>>>((float*)x, pos, tokens, H, D); },
       [&] { rope_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((__nv_bfloat16*)x, pos, tokens, H, D); });

@@ -515,10 +515,19 @@ pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual,
     PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
   PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, static_cast<cudaStream_t>(stream)));
 }
+pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
+                                    int32_t k, int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, w_gate, w_up, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
+  if (m == 0) return PYR_OK;
+  if (dtype != PYR_BF16 || !pyr::gemm_tc_supported(x, w_gate, w_up, out, m, n, k)) return PYR_ERR_UNSUPPORTED;
+  PYR_GLUE(pyr::launch_gemm_tc_gated(x, w_gate, w_up, out, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
+}
 pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,
                            int32_t dtype, void* stream) {
   if (!glue_ok(dtype, {x, pos})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
   if (tokens < 0 || n_heads < 1 || head_dim < 2 || head_dim % 2) return PYR_ERR_INVALID;
+  if (head_dim > 256) return PYR_ERR_UNSUPPORTED;
   PYR_GLUE(pyr::launch_glue_rope(x, pos, tokens, n_heads, head_dim, dtype, static_cast<cudaStream_t>(stream)));
 }
 pyr_status_t pyr_glue_swiglu(const void* gate, const void* up, void* out, int64_t n, int32_t dtype, void* stream) {

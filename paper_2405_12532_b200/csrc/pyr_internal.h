@@ -120,6 +120,8 @@ cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, vo
 bool gemm_tc_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
 cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
                            cudaStream_t s);
+cudaError_t launch_gemm_tc_gated(const void* x, const void* wg, const void* wu, void* out, int64_t M, int N, int K,
+                                 int* status, cudaStream_t s);
 bool gemm_skinny_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
 cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
                                cudaStream_t s);

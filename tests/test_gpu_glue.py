@@ -91,3 +91,31 @@ def test_skinny_linear_whole_output(M, N, K, res):
         want = want + r.double()
     scale = float(want.abs().max().clamp_min(1e-3))
     assert float((y.double() - want).abs().max()) <= 2 ** -7 * scale
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 512, 256), (4096, 11008, 4096), (129, 1000, 64), (65, 128, 128)])
+def test_gated_linear_against_fp64(M, N, K):
+    """pyr_glue_linear_swiglu: silu(x wg^T) * (x wu^T) from the fp32 accumulators, against fp64 on sampled
+    entries and one whole row; fp32 and unaligned shapes are refused."""
+    x = _r(M, K, seed=41, dtype=torch.bfloat16)
+    wg = (_r(N, K, seed=42) * 0.05).to(torch.bfloat16)
+    wu = (_r(N, K, seed=43) * 0.05).to(torch.bfloat16)
+    launches = pb.launch_count()
+    out = pb.glue_linear_swiglu(x, wg, wu)
+    torch.cuda.synchronize()
+    assert pb.launch_count() - launches == 1
+    rng = np.random.default_rng(M + N)
+    rows = np.concatenate([[0, M - 1, min(127, M - 1), min(128, M - 1)], rng.integers(0, M, size=60)])
+    cols = np.concatenate([[0, N - 1, min(127, N - 1), min(128, N - 1)], rng.integers(0, N, size=60)])
+    rt, ct = torch.from_numpy(rows).to(DEV), torch.from_numpy(cols).to(DEV)
+    g = (x[rt].double() * wg[ct].double()).sum(-1)
+    u = (x[rt].double() * wu[ct].double()).sum(-1)
+    want = g / (1 + torch.exp(-g)) * u
+    got = out[rt, ct].double()
+    scale = float(want.abs().max().clamp_min(1e-3))
+    assert float((got - want).abs().max()) <= 2 ** -7 * scale
+    gr = synth.widen(x[M // 2]) @ synth.widen(wg).T
+    ur = synth.widen(x[M // 2]) @ synth.widen(wu).T
+    np.testing.assert_allclose(synth.widen(out[M // 2]), gr / (1 + np.exp(-gr)) * ur, atol=2 ** -7 * scale, rtol=2 ** -7)
+    with pytest.raises(Exception):
+        pb.glue_linear_swiglu(x.float(), wg.float(), wu.float())

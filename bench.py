@@ -258,8 +258,9 @@ class Workload:
 class ModelWorkload(Workload):
     """The 7B-shaped workload as a whole model on the library's kernels: embedding, RMSNorm, the
     projections and the MLP on the tcgen05 GEMM, rotary embedding at original positions, the pyramid
-    path, o_proj on all rows followed by the in-place compaction of the hidden rows, greedy head.
-    torch holds the tensors (and makes the compacted rows contiguous between layers)."""
+    path, o_proj on all rows, then the MLP on the kept rows read where they lie (the hidden states are
+    never compacted: the norm and the residual of the down projection go through the kept list),
+    greedy head. torch holds the tensors."""
 
     def __init__(self, name: str, device, layers: int = 0, decode_steps: int = -1, batch: int = 0, reselect_every: int = 0):
         from paper_2405_12532_b200 import binding as pb
@@ -318,13 +319,14 @@ class ModelWorkload(Workload):
             y = pb.glue_linear(o.view(B, n, d), W[f"wo{l}"], x)
             if events is not None:
                 events[l][1].record()
-            n_out = c.select_compact(l, k, v, y, d, n * d, d, 0)
+            c.select_compact(l, k, v, None, 0, 0, 0, 0)      # K/V into the cache, kept list, positions; y stays where it is
             if events is not None:
                 events[l][2].record()
-            y = y[:, :n_out].contiguous()
-            pos = c.kept(l)[1][:, 0].contiguous()
-            h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
-            x = pb.glue_linear(pb.glue_linear_swiglu(h2, W[f"wg{l}"], W[f"wu{l}"]), W[f"wd{l}"], y)
+            kept, kept_pos = c.kept(l)
+            rows = kept[:, 0]                                # [B, n_out]: the kept rows of every sequence
+            pos = kept_pos[:, 0].contiguous()
+            h2 = pb.glue_rmsnorm_rows(y, rows, W[f"n2{l}"])
+            x = pb.glue_linear_rows(pb.glue_linear_swiglu(h2, W[f"wg{l}"], W[f"wu{l}"]), W[f"wd{l}"], y, rows)
         logits = pb.glue_linear(pb.glue_rmsnorm(x[:, -1].contiguous(), W["nf"]), W["head"])
         self.first_token = pb.glue_argmax(logits)
 

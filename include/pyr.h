@@ -324,6 +324,13 @@ pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
  *           and n a multiple of 128 a weight-streaming kernel whose clusters split k and add their
  *           partial sums in a fixed order, else a tiled kernel (n a multiple of 8). Results are
  *           bit-reproducible run to run in every case. Everything else takes the CUDA-core kernel.
+ *   rmsnorm_rows / linear_rows  the same two operations reading through a list of rows per sequence,
+ *           so that kept rows are used where they lie and the hidden states are never compacted:
+ *           rmsnorm_rows: out[b, i, :] = rmsnorm(x[b, rows[b * rows_stride + i], :]) for x [batch, n_src, d],
+ *           out [batch, n_dst, d]; linear_rows: y[b, i, :] = x[b, i, :] . w^T + residual[b, res_rows[b *
+ *           rows_stride + i], :] for x [batch, n_dst, k], residual [batch, n_src, n], y [batch, n_dst, n].
+ *           The lists are device int32 (pyr_cache_kept's first pointer, a dense [B, n_out] array when
+ *           sel_groups == 1: rows_stride = n_out); their entries must lie in [0, n_src), which is not checked.
  *   linear_swiglu  out[m, n] = silu(x . w_gate^T) * (x . w_up^T), w_gate and w_up [n, k]: the gated MLP's
  *           first half in one pass, neither projection written out (fp32 accumulators go straight
  *           into the product). bf16 with 16-byte aligned pointers, k a multiple of 64 and n a
@@ -341,6 +348,12 @@ pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_
                               int32_t dtype, void* stream);
 pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual, void* y, int64_t m, int32_t n,
                              int32_t k, int32_t dtype, void* stream);
+pyr_status_t pyr_glue_rmsnorm_rows(const void* x, const int32_t* rows, int64_t rows_stride, const void* gain, void* out,
+                                   int32_t batch, int32_t n_src, int32_t n_dst, int32_t d, float eps, int32_t dtype,
+                                   void* stream);
+pyr_status_t pyr_glue_linear_rows(const void* x, const void* w, const void* residual, const int32_t* res_rows,
+                                  int64_t rows_stride, void* y, int32_t batch, int32_t n_src, int32_t n_dst, int32_t n,
+                                  int32_t k, int32_t dtype, void* stream);
 pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
                                     int32_t k, int32_t dtype, void* stream);
 pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,

@@ -25,7 +25,7 @@ PYR_FLAG_POS_REENCODE = 4
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_swiglu",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_swiglu", "pyr_glue_rmsnorm_rows", "pyr_glue_linear_rows",
     "pyr_glue_rope", "pyr_glue_swiglu", "pyr_glue_argmax", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
         L.pyr_glue_rmsnorm.argtypes = [vp, vp, vp, i64, i32, C.c_float, i32, vp]
         L.pyr_glue_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
         L.pyr_glue_linear_swiglu.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
+        L.pyr_glue_rmsnorm_rows.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, C.c_float, i32, vp]
+        L.pyr_glue_linear_rows.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i32, i32, i32, i32, vp]
         L.pyr_glue_rope.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.pyr_glue_swiglu.argtypes = [vp, vp, vp, i64, i32, vp]
         L.pyr_glue_argmax.argtypes = [vp, vp, i64, i32, i32, vp]
@@ -195,6 +197,30 @@ def glue_linear(x, w, residual=None):
     y = torch.empty(*x.shape[:-1], N, dtype=x.dtype, device=x.device)
     _check(lib().pyr_glue_linear(x.data_ptr(), w.data_ptr(), residual.data_ptr() if residual is not None else None,
                                  y.data_ptr(), x.numel() // K, N, K, _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_linear")
+    return y
+
+
+def glue_rmsnorm_rows(x, rows, gain, eps: float = 1e-5):
+    """rmsnorm of the rows rows[b, i] of x [B, n_src, d] -> [B, n_dst, d] (pyr_glue_rmsnorm_rows); rows int32 [B, n_dst], last dim contiguous."""
+    assert x.is_contiguous() and x.dim() == 3 and rows.dtype == torch.int32 and rows.dim() == 2 and rows.stride(1) == 1
+    B, n_src, d = x.shape
+    n_dst = rows.shape[1]
+    out = torch.empty(B, n_dst, d, dtype=x.dtype, device=x.device)
+    _check(lib().pyr_glue_rmsnorm_rows(x.data_ptr(), rows.data_ptr(), rows.stride(0), gain.data_ptr(), out.data_ptr(), B, n_src, n_dst, d,
+                                       float(eps), _dt(x), C.c_void_p(_stream_ptr(None))), "pyr_glue_rmsnorm_rows")
+    return out
+
+
+def glue_linear_rows(x, w, residual, res_rows):
+    """x [B, n_dst, K] . w [N, K]^T + residual[b, res_rows[b, i]] for residual [B, n_src, N] -> [B, n_dst, N] (pyr_glue_linear_rows)."""
+    assert x.is_contiguous() and w.is_contiguous() and residual.is_contiguous() and x.dim() == 3 and residual.dim() == 3
+    assert res_rows.dtype == torch.int32 and res_rows.dim() == 2 and res_rows.stride(1) == 1 and res_rows.shape[1] == x.shape[1]
+    N, K = w.shape
+    B, n_dst, _ = x.shape
+    y = torch.empty(B, n_dst, N, dtype=x.dtype, device=x.device)
+    _check(lib().pyr_glue_linear_rows(x.data_ptr(), w.data_ptr(), residual.data_ptr(), res_rows.data_ptr(), res_rows.stride(0),
+                                      y.data_ptr(), B, residual.shape[1], n_dst, N, K, _dt(x), C.c_void_p(_stream_ptr(None))),
+           "pyr_glue_linear_rows")
     return y
 
 

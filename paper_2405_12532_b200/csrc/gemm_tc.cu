@@ -52,6 +52,7 @@ struct GemmArgs {
   int64_t M;
   int N, K;
   int* status;                // may be null
+  RowMap res_map;             // rows of `res` that the rows of y add (identity when its list is null)
 };
 
 __device__ __forceinline__ void tile_of(int tile, int mblocks, int nblocks, int* mb, int* nb) {
@@ -188,7 +189,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int n = n0 + c32 * 32;
         if (m < a.M && n < a.N) {                 // N is a multiple of 8: whole 16-byte chunks are in or out
           __nv_bfloat16* yp = a.y + m * a.N + n;
-          const __nv_bfloat16* rp = a.res ? a.res + m * a.N + n : nullptr;
+          const __nv_bfloat16* rp = a.res ? a.res + a.res_map.source_row(m) * a.N + n : nullptr;
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             if (n + ch * 8 < a.N) {
@@ -243,7 +244,7 @@ bool gemm_tc_supported(const void* x, const void* w, const void* res, const void
 }
 
 cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
-                           cudaStream_t s) {
+                           const RowMap& res_map, cudaStream_t s) {
   const int sms = device_sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   // wide tiles when there are enough of them to fill the machine, else narrower ones
@@ -255,7 +256,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* 
     return cudaErrorInvalidValue;
   GemmArgs a;
   a.res = static_cast<const __nv_bfloat16*>(res); a.y = static_cast<__nv_bfloat16*>(y);
-  a.M = M; a.N = N; a.K = K; a.status = status;
+  a.M = M; a.N = N; a.K = K; a.status = status; a.res_map = res_map;
   return BN == 256 ? run_gemm<256, false>(mx, mw, mw, a, sms, s) : run_gemm<128, false>(mx, mw, mw, a, sms, s);
 }
 

@@ -29,11 +29,14 @@ __global__ void embed_kernel(const int32_t* ids, const T* table, T* out, int64_t
   for (int i = threadIdx.x; i < d; i += blockDim.x) out[t * d + i] = table[(int64_t)id * d + i];
 }
 
-// out = x / sqrt(mean(x^2) + eps) * gain, one CTA per row, the squares summed in a fixed order
+// out = x / sqrt(mean(x^2) + eps) * gain, one CTA per row, the squares summed in a fixed order.
+// With a row map, output row (b, i) reads x row (b, rows[b][i]): the kept rows are normalised
+// straight out of the uncompacted tensor.
 template <typename T>
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const T* x, const T* gain, T* out, int d, float eps) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const T* x, const T* gain, T* out, int d, float eps, RowMap map) {
   __shared__ float red[8];
   const int64_t t = blockIdx.x;
+  x += (map.source_row(t) - t) * d;
   float s = 0.f;
   for (int i = threadIdx.x; i < d; i += 256) { const float v = ld(x + t * d + i); s = fmaf(v, v, s); }
 #pragma unroll
@@ -49,7 +52,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const T* x, const T* gain,
 
 // y[t, n] = sum_k x[t, k] w[n, k] (+ res[t, n]); 64 x 64 output tile per CTA, 16 k per step, 4 x 4 outputs per thread
 template <typename T>
-__global__ void __launch_bounds__(256) linear_kernel(const T* x, const T* w, const T* res, T* y, int64_t M, int N, int K) {
+__global__ void __launch_bounds__(256) linear_kernel(const T* x, const T* w, const T* res, T* y, int64_t M, int N, int K,
+                                                     RowMap map) {
   __shared__ float xs[16][64 + 1], ws[16][64 + 1];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int64_t m0 = (int64_t)blockIdx.y * 64;
@@ -80,7 +84,7 @@ __global__ void __launch_bounds__(256) linear_kernel(const T* x, const T* w, con
     for (int j = 0; j < 4; ++j) {
       const int64_t m = m0 + ty * 4 + i;
       const int n = n0 + tx * 4 + j;
-      if (m < M && n < N) st(y + m * N + n, acc[i][j] + (res ? ld(res + m * N + n) : 0.f));
+      if (m < M && n < N) st(y + m * N + n, acc[i][j] + (res ? ld(res + map.source_row(m) * N + n) : 0.f));
     }
 }
 
@@ -160,19 +164,19 @@ cudaError_t launch_glue_embed(const int32_t* ids, const void* table, void* out, 
       [&] { embed_kernel<__nv_bfloat16><<<(unsigned)tokens, 128, 0, s>>>(ids, (const __nv_bfloat16*)table, (__nv_bfloat16*)out, tokens, d, vocab, status); });
 }
 cudaError_t launch_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int d, float eps, int dtype,
-                                cudaStream_t s) {
+                                const RowMap& map, cudaStream_t s) {
   if (tokens == 0) return cudaSuccess;
   return by_dtype(dtype,
-      [&] { rmsnorm_kernel<float><<<(unsigned)tokens, 256, 0, s>>>((const float*)x, (const float*)gain, (float*)out, d, eps); },
-      [&] { rmsnorm_kernel<__nv_bfloat16><<<(unsigned)tokens, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, d, eps); });
+      [&] { rmsnorm_kernel<float><<<(unsigned)tokens, 256, 0, s>>>((const float*)x, (const float*)gain, (float*)out, d, eps, map); },
+      [&] { rmsnorm_kernel<__nv_bfloat16><<<(unsigned)tokens, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, d, eps, map); });
 }
 cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int dtype,
-                               cudaStream_t s) {
+                               const RowMap& map, cudaStream_t s) {
   if (M == 0 || N == 0) return cudaSuccess;
   dim3 grid((N + 63) / 64, (unsigned)((M + 63) / 64));
   return by_dtype(dtype,
-      [&] { linear_kernel<float><<<grid, 256, 0, s>>>((const float*)x, (const float*)w, (const float*)res, (float*)y, M, N, K); },
-      [&] { linear_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, (const __nv_bfloat16*)res, (__nv_bfloat16*)y, M, N, K); });
+      [&] { linear_kernel<float><<<grid, 256, 0, s>>>((const float*)x, (const float*)w, (const float*)res, (float*)y, M, N, K, map); },
+      [&] { linear_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, (const __nv_bfloat16*)res, (__nv_bfloat16*)y, M, N, K, map); });
 }
 cudaError_t launch_glue_rope(void* x, const int32_t* pos, int64_t tokens, int H, int D, int dtype, cudaStream_t s) {
   if (tokens == 0) return cudaSuccess;

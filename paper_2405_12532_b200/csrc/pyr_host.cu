@@ -498,11 +498,31 @@ pyr_status_t pyr_glue_embed(const int32_t* ids, const void* table, void* out, in
   if (tokens < 0 || d < 1 || vocab < 1) return PYR_ERR_INVALID;
   PYR_GLUE(pyr::launch_glue_embed(ids, table, out, tokens, d, vocab, dtype, dev_status, static_cast<cudaStream_t>(stream)));
 }
+namespace {
+// a row list per sequence: every argument in range, the list's rows themselves are the caller's promise
+bool row_map_ok(const int32_t* rows, int32_t batch, int32_t n_src, int32_t n_dst, int64_t rows_stride) {
+  return rows && batch >= 0 && n_src >= 1 && n_dst >= 1 && rows_stride >= n_dst;
+}
+pyr::RowMap row_map(const int32_t* rows, int32_t n_src, int32_t n_dst, int64_t rows_stride) {
+  pyr::RowMap m;
+  m.rows = rows; m.rows_stride = rows_stride; m.n_src = n_src; m.n_dst = n_dst;
+  return m;
+}
+}  // namespace
+
 pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int32_t d, float eps,
                               int32_t dtype, void* stream) {
   if (!glue_ok(dtype, {x, gain, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
   if (tokens < 0 || d < 1 || !(eps >= 0.f)) return PYR_ERR_INVALID;
-  PYR_GLUE(pyr::launch_glue_rmsnorm(x, gain, out, tokens, d, eps, dtype, static_cast<cudaStream_t>(stream)));
+  PYR_GLUE(pyr::launch_glue_rmsnorm(x, gain, out, tokens, d, eps, dtype, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_rmsnorm_rows(const void* x, const int32_t* rows, int64_t rows_stride, const void* gain, void* out,
+                                   int32_t batch, int32_t n_src, int32_t n_dst, int32_t d, float eps, int32_t dtype,
+                                   void* stream) {
+  if (!glue_ok(dtype, {x, rows, gain, out})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (!row_map_ok(rows, batch, n_src, n_dst, rows_stride) || d < 1 || !(eps >= 0.f)) return PYR_ERR_INVALID;
+  PYR_GLUE(pyr::launch_glue_rmsnorm(x, gain, out, (int64_t)batch * n_dst, d, eps, dtype, row_map(rows, n_src, n_dst, rows_stride),
+                                    static_cast<cudaStream_t>(stream)));
 }
 pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual, void* y, int64_t m, int32_t n,
                              int32_t k, int32_t dtype, void* stream) {
@@ -512,8 +532,20 @@ pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual,
   if (dtype == PYR_BF16 && pyr::gemm_skinny_supported(x, w, residual, y, m, n, k))
     PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
   if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
-    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
-  PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, static_cast<cudaStream_t>(stream)));
+    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
+  PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_linear_rows(const void* x, const void* w, const void* residual, const int32_t* res_rows,
+                                  int64_t rows_stride, void* y, int32_t batch, int32_t n_src, int32_t n_dst, int32_t n,
+                                  int32_t k, int32_t dtype, void* stream) {
+  if (!glue_ok(dtype, {x, w, residual, res_rows, y})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (!row_map_ok(res_rows, batch, n_src, n_dst, rows_stride) || n < 1 || k < 1) return PYR_ERR_INVALID;
+  const int64_t m = (int64_t)batch * n_dst;
+  if (m == 0) return PYR_OK;
+  const pyr::RowMap map = row_map(res_rows, n_src, n_dst, rows_stride);
+  if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
+    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, map, static_cast<cudaStream_t>(stream)));
+  PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, map, static_cast<cudaStream_t>(stream)));
 }
 pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
                                     int32_t k, int32_t dtype, void* stream) {

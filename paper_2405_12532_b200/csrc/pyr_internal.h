@@ -112,14 +112,29 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t s);
 // decoder glue of whole-model workloads (csrc/glue.cu); matrices row-major, w is [N, K] (out, in)
 cudaError_t launch_glue_embed(const int32_t* ids, const void* table, void* out, int64_t tokens, int d, int vocab,
                               int dtype, int* status, cudaStream_t s);
+// Rows of a [batch, n_src, *] tensor picked by a list per sequence: logical row b * n_dst + i is physical row
+// b * n_src + rows[b * rows_stride + i]. rows == nullptr: the identity.
+struct RowMap {
+  const int32_t* rows = nullptr;
+  int64_t rows_stride = 0;
+  int n_src = 0, n_dst = 1;
+#ifdef __CUDACC__
+  __host__ __device__
+#endif
+  int64_t source_row(int64_t m) const {
+    if (!rows) return m;
+    const int64_t b = m / n_dst;
+    return b * n_src + rows[b * rows_stride + (m - b * n_dst)];
+  }
+};
 cudaError_t launch_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int d, float eps, int dtype,
-                                cudaStream_t s);
+                                const RowMap& map, cudaStream_t s);
 cudaError_t launch_glue_linear(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int dtype,
-                               cudaStream_t s);
+                               const RowMap& map, cudaStream_t s);
 // bf16 tensor-core GEMM of the glue (csrc/gemm_tc.cu): y = x w^T (+ res); w is [N, K]
 bool gemm_tc_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
 cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
-                           cudaStream_t s);
+                           const RowMap& res_map, cudaStream_t s);
 cudaError_t launch_gemm_tc_gated(const void* x, const void* wg, const void* wu, void* out, int64_t M, int N, int K,
                                  int* status, cudaStream_t s);
 bool gemm_skinny_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);

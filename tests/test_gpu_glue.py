@@ -119,3 +119,35 @@ def test_gated_linear_against_fp64(M, N, K):
     np.testing.assert_allclose(synth.widen(out[M // 2]), gr / (1 + np.exp(-gr)) * ur, atol=2 ** -7 * scale, rtol=2 ** -7)
     with pytest.raises(Exception):
         pb.glue_linear_swiglu(x.float(), wg.float(), wu.float())
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-5), (torch.bfloat16, 2 ** -7)])
+def test_row_mapped_norm_and_residual(dtype, tol):
+    """pyr_glue_rmsnorm_rows / pyr_glue_linear_rows read kept rows where they lie: equal to gathering first."""
+    B, n_src, n_dst, d, N = 3, 300, 170, 256, 384
+    g = torch.Generator().manual_seed(5)
+    rows = torch.stack([torch.sort(torch.randperm(n_src, generator=g)[:n_dst]).values for _ in range(B)]).to(torch.int32)
+    pad = torch.full((B, 7), -1, dtype=torch.int32)                       # a list stride wider than n_dst
+    rows_dev = torch.cat([rows, pad], 1).to(DEV)[:, :n_dst]
+    x = _r(B, n_src, d, seed=51, dtype=dtype)
+    gain = _r(d, seed=52, dtype=dtype)
+    gathered = torch.gather(x, 1, rows.to(DEV).long()[:, :, None].expand(B, n_dst, d)).contiguous()
+    got = pb.glue_rmsnorm_rows(x, rows_dev, gain)
+    assert torch.equal(got, pb.glue_rmsnorm(gathered, gain))
+    h = _r(B, n_dst, d, seed=53, dtype=dtype)
+    w = (_r(N, d, seed=54) * 0.05).to(dtype)
+    res = _r(B, n_src, N, seed=55, dtype=dtype)
+    res_g = torch.gather(res, 1, rows.to(DEV).long()[:, :, None].expand(B, n_dst, N)).contiguous()
+    y = pb.glue_linear_rows(h, w, res, rows_dev)
+    assert torch.equal(y, pb.glue_linear(h, w, res_g))
+    want = synth.widen(h) @ synth.widen(w).T + synth.widen(res_g)
+    np.testing.assert_allclose(synth.widen(y), want, atol=tol * float(np.abs(want).max()), rtol=tol)
+    # a bigger bf16 case that takes the tensor-core kernel
+    if dtype == torch.bfloat16:
+        B2, s2, d2, k2 = 2, 900, 700, 512
+        rows2 = torch.stack([torch.sort(torch.randperm(s2, generator=g)[:d2]).values for _ in range(B2)]).to(torch.int32).to(DEV)
+        h2 = _r(B2, d2, k2, seed=56, dtype=dtype)
+        w2 = (_r(1024, k2, seed=57) * 0.05).to(dtype)
+        r2 = _r(B2, s2, 1024, seed=58, dtype=dtype)
+        r2g = torch.gather(r2, 1, rows2.long()[:, :, None].expand(B2, d2, 1024)).contiguous()
+        assert torch.equal(pb.glue_linear_rows(h2, w2, r2, rows2), pb.glue_linear(h2, w2, r2g))

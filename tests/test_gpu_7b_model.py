@@ -120,6 +120,20 @@ def test_7b_shaped_model_batch1_all_layers():
         if l in checked:
             _check_linear(ok, W[f"wo{l}"], y, rng, res=xk)
             _check_linear(act, W[f"wd{l}"], x, rng, res=y)
+            # the gated GEMM (gate, up and SwiGLU in one pass) on the same input, against fp64 on sampled entries
+            act_f = pb.glue_linear_swiglu(h2, W[f"wg{l}"], W[f"wu{l}"]).view(-1, FF)
+            rr = torch.from_numpy(rng.integers(0, act_f.shape[0], size=24)).to(DEV)
+            cc = torch.from_numpy(rng.integers(0, FF, size=24)).to(DEV)
+            gg = (h2.view(-1, HID)[rr].double() * W[f"wg{l}"][cc].double()).sum(-1)
+            uu = (h2.view(-1, HID)[rr].double() * W[f"wu{l}"][cc].double()).sum(-1)
+            want = gg / (1 + torch.exp(-gg)) * uu
+            assert float((act_f[rr, cc].double() - want).abs().max()) <= 2 ** -7 * float(want.abs().max().clamp_min(1e-3)) + 1e-4
+            # the MLP read through the kept list from uncompacted rows equals the MLP of the compacted rows
+            y_all = torch.zeros(B, n, HID, dtype=y.dtype, device=DEV)
+            y_all[0, idx] = y[0]
+            assert torch.equal(pb.glue_rmsnorm_rows(y_all, kept[:, 0], W[f"n2{l}"]), h2)
+            assert torch.equal(pb.glue_linear_rows(act, W[f"wd{l}"], y_all, kept[:, 0]), x)
+            del act_f, y_all
         pos = posk[:, 0].contiguous()
         del q, kk, v, o, rows_t, h, h2, act, y
     logits = pb.glue_linear(pb.glue_rmsnorm(x[:, -1].contiguous(), W["nf"]), W["head"])

@@ -180,3 +180,32 @@ def test_max_batch_under_a_memory_cap_table2_shape():
     pyr = max_batch(synth.ratio_schedule(w), 16)
     assert 60 <= full <= 90             # 2 * 40 layers * 5120 * 2 B * 768 rows = 0.63 GB per sequence
     assert pyr / full > 1.8
+
+
+def test_glue_entry_points_validate_before_any_launch():
+    """The decoder-glue calls refuse bad arguments on the host: null pointers, unknown dtypes, sizes out
+    of range, and the shapes the fused forms do not cover - none of which reaches a kernel launch."""
+    L = pb.lib()
+    P = C.c_void_p(FAKE_DEV)
+    NULL = C.c_void_p(None)
+    i64, i32, f32 = C.c_int64, C.c_int32, C.c_float
+    L.pyr_glue_linear.restype = L.pyr_glue_rope.restype = L.pyr_glue_linear_swiglu.restype = C.c_int
+    L.pyr_glue_rmsnorm_rows.restype = L.pyr_glue_linear_rows.restype = C.c_int
+    assert L.pyr_glue_linear(NULL, P, NULL, P, i64(4), i32(8), i32(8), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear(P, P, NULL, P, i64(4), i32(0), i32(8), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_linear(P, P, NULL, P, i64(4), i32(8), i32(8), i32(9), NULL) == pb.PYR_ERR_UNSUPPORTED
+    assert L.pyr_glue_linear(P, P, NULL, P, i64(0), i32(8), i32(8), i32(pb.PYR_BF16), NULL) == pb.PYR_OK      # nothing to do
+    # the gated form: bf16, k a multiple of 64, n a multiple of 8
+    assert L.pyr_glue_linear_swiglu(P, P, NULL, P, i64(4), i32(8), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear_swiglu(P, P, P, P, i64(4), i32(8), i32(64), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_UNSUPPORTED
+    assert L.pyr_glue_linear_swiglu(P, P, P, P, i64(4), i32(8), i32(48), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_UNSUPPORTED
+    assert L.pyr_glue_linear_swiglu(P, P, P, P, i64(-1), i32(8), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_INVALID
+    # rotary embedding: even head_dim up to 256
+    assert L.pyr_glue_rope(P, P, i64(4), i32(2), i32(7), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_rope(P, P, i64(4), i32(2), i32(512), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_UNSUPPORTED
+    # row lists: a list stride shorter than the list, empty sources
+    assert L.pyr_glue_rmsnorm_rows(P, P, i64(3), P, P, i32(2), i32(10), i32(4), i32(16), f32(1e-5), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_rmsnorm_rows(P, NULL, i64(4), P, P, i32(2), i32(10), i32(4), i32(16), f32(1e-5), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(2), i32(0), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_linear_rows(P, P, NULL, P, i64(4), P, i32(2), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(0), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_OK

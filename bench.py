@@ -488,7 +488,10 @@ def run_ours(args, rank, world, local_rank, workload=None):
     # attention-path numbers of the headline line
     model = None
     if name == DEFAULT_WORKLOAD and not args.no_model and not (args.layers or args.batch or args.decode_steps >= 0):
-        model = run_model(args, rank, world, local_rank, MODEL_WORKLOAD, emit=False)
+        # an auxiliary figure: a few steps are enough, however long the headline run is asked to be
+        margs = argparse.Namespace(**vars(args))
+        margs.steps, margs.warmup = min(args.steps, 5), min(args.warmup, 3)
+        model = run_model(margs, rank, world, local_rank, MODEL_WORKLOAD, emit=False)
 
     if rank != 0:
         return
@@ -549,6 +552,7 @@ def run_ours(args, rank, world, local_rank, workload=None):
         line["whole_model"] = {k: model[k] for k in ("value", "unit", "decode_tokens_per_s", "ms_prefill", "ms_decode",
                                                       "roofline", "roofline_decode", "gpu_launches", "clocks")}
         line["whole_model"]["workload"] = MODEL_WORKLOAD
+        line["whole_model"]["steps"], line["whole_model"]["warmup"] = model["steps"], model["warmup"]
     print(json.dumps(line), flush=True)
 
 

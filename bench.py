@@ -126,7 +126,7 @@ class Workload:
     """Device-resident synthetic inputs and the call sequence of one step."""
 
     def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1, batch: int = 0,
-                 reselect_every: int = 0):
+                 reselect_every: int = 0, select_first: bool = False):
         from paper_2405_12532_b200 import binding as pb
         self.pb = pb
         self.name = name
@@ -142,6 +142,12 @@ class Workload:
             w["batch"] = batch
         self.reselect_every = reselect_every      # generation-phase PvC update every so many decode steps (0: never)
         flags = pb.PYR_FLAG_GEN_RESELECT if reselect_every else 0
+        # Select-first ordering (on request) where the rows that select + compact moves are the attention output itself
+        # (one kept set per head group): the kept rows are then written in place by the attention kernel. With one
+        # kept set per sequence the compacted rows are the hidden states, which attention does not produce.
+        self.select_first = bool(select_first and w["sel_groups"] > 1 and w["dtype"] == "bf16" and w["head_dim"] == 128)
+        if self.select_first:
+            flags |= pb.PYR_FLAG_SELECT_FIRST
         self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio, flags=flags))
         self.layers = [self.cache.layer_info(l) for l in range(w["n_layers"])]
         B, N, Hq, Hkv, D = w["batch"], w["prompt_len"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
@@ -240,7 +246,10 @@ class Workload:
             tot += 2 * 2 * B * Hkv * n_out * D * self.eb                    # K and V, read + write
             if n_out < n:
                 row_b = (self.hidden if G == 1 else (w["n_q_heads"] // Hkv) * D) * self.eb
-                tot += 2 * B * G * n_out * row_b                            # compacted rows, read + write
+                # select-first ordering: only the window's rows (and the few kept rows of the tile that holds the
+                # window's start, not counted here) are still moved; the others were written in place
+                moved = min(Lw, n) if (self.select_first and c > 0) else n_out
+                tot += 2 * B * G * moved * row_b                            # compacted rows, read + write
             tot += 2 * B * G * n_out * 4                                    # positions
         return tot
 
@@ -438,7 +447,7 @@ def run_ours(args, rank, world, local_rank, workload=None):
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
     wl = Workload(name, device, layers=args.layers, decode_steps=args.decode_steps, batch=args.batch,
-                  reselect_every=args.reselect_every)
+                  reselect_every=args.reselect_every, select_first=args.select_first)
     w = wl.w
     nL = w["n_layers"]
     hbm, tf_burst, tf_sust, peak_src = measured_peaks()
@@ -542,6 +551,8 @@ def run_ours(args, rank, world, local_rank, workload=None):
                    "heads": w["n_q_heads"], "kv_heads": w["n_kv_heads"], "head_dim": w["head_dim"],
                    "ratio": "geometric 1.0->%.2f" % wl.ratio[-1],
                    "reselect_every": args.reselect_every or None,
+                   "ordering": ("select-first: the window's query tiles, scores and selection, then the other tiles writing "
+                                "kept rows in place (the selection is timed with the attention)") if wl.select_first else "default",
                    "l2": "inputs larger than L2 (each of Q, K, V and the cache is >= 1 GB)"},
         "roofline": dominant, "roofline_prefill": roof_pre, "roofline_select_compact": roof_sel,
         "roofline_decode": roof_dec,
@@ -757,6 +768,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--select-first", action="store_true",
+                    help="select-first ordering on the per-head workloads: the window's query tiles, the scores and the "
+                         "selection first, then the other tiles writing kept rows in place")
     ap.add_argument("--no-model", action="store_true", help="skip the whole-model run that the default workload reports beside its line")
     ap.add_argument("--reselect-every", type=int, default=0,
                     help="generation-phase PvC update of every layer every so many decode steps (0: never)")

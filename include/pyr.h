@@ -76,6 +76,15 @@ typedef enum { PYR_BF16 = 0, PYR_F32 = 1 } pyr_dtype_t;
                                          original positions), which the paper finds slightly better */
 #define PYR_FLAG_GEN_RESELECT 2u      /* keep each layer's recent queries so that pyr_decode_reselect can
                                          update the PvC during generation (Section 4.1, Generation Phase) */
+#define PYR_FLAG_SELECT_FIRST 8u      /* select-first ordering (bf16, head_dim 128): pyr_prefill_layer computes the
+                                         query tiles that hold the recent window, the scores and the selection
+                                         first, then the remaining query tiles, writing each kept row of `out`
+                                         straight to its place among the kept rows of its selection group (dropped
+                                         rows are not written). pyr_select_compact then gathers K/V and, when its
+                                         `rows` is that same `out`, only moves the rows of the first tiles down;
+                                         any other `rows` is compacted in full as always. The results equal the
+                                         default ordering's. Layers that drop nothing, and configurations the
+                                         tensor-core kernels do not cover, take the default ordering. */
 
 /*
  * Parameters of Algorithm 1 (recent window length L, minimum PvC lengths N_l,

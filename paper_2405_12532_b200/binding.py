@@ -21,6 +21,7 @@ PYR_BF16, PYR_F32 = 0, 1
 PYR_FLAG_CUDA_CORE_PREFILL = 1
 PYR_FLAG_GEN_RESELECT = 2
 PYR_FLAG_POS_REENCODE = 4
+PYR_FLAG_SELECT_FIRST = 8
 
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",

@@ -82,10 +82,12 @@ struct Tile {
 // A head's tiles can be dealt to `parts` CTAs. With the tiles numbered from the longest (k = 0),
 // part p takes k = p, 2 parts - 1 - p, 2 parts + p, 4 parts - 1 - p, ...: a long tile is paired with
 // a short one, so the parts carry nearly equal work. Returns false when the part has no it-th tile.
-__host__ __device__ __forceinline__ bool tile_at(int it, int part, int parts, int n, Tile* tl) {
+// A launch may cover only the tiles k0 <= k < k1 (select-first ordering: the tiles that hold the
+// recent window first, the rest once the kept rows are known).
+__host__ __device__ __forceinline__ bool tile_at(int it, int part, int parts, int n, int k0, int k1, Tile* tl) {
   const int ntiles = (n + kTile - 1) / kTile;
-  const int k = 2 * parts * (it >> 1) + ((it & 1) ? 2 * parts - 1 - part : part);
-  if (k >= ntiles) return false;
+  const int k = k0 + 2 * parts * (it >> 1) + ((it & 1) ? 2 * parts - 1 - part : part);
+  if (k >= ntiles || k >= k1) return false;
   const int ti = ntiles - 1 - k;
   tl->r0 = ti * kTile;
   tl->nkt = ti + 1;
@@ -186,9 +188,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint8_t* my_row = sm.o_stage + row * 128;
     bool ok = true, stored = false;
     int ring0 = 0;
+    // select-first ordering: rows leave for their place among the kept rows of the head's selection group
+    const int32_t* rank = a.rank ? a.rank + ((int64_t)b * a.G + (a.G == 1 ? 0 : h / (a.Hq / a.G))) * n : nullptr;
+    __nv_bfloat16* out_bh = static_cast<__nv_bfloat16*>(a.out) + (int64_t)b * a.osb + (int64_t)h * a.osh;
     for (int it = 0;; ++it) {
       Tile tl;
-      if (!tile_at(it, part, parts, n, &tl)) break;
+      if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;
       const int nkt = tl.nkt;
       const int i = tl.r0 + row;
       const int gf = (ring0 + nkt - 1) & 1;               // the group that took the tile's last K tile
@@ -207,6 +212,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_fin + log2f(l)) * kLn2;
       const float inv = 1.f / l;
+
       // O leaves through shared memory, one [128 x 64] half at a time (rows past n are clipped by the store)
 #pragma unroll 1
       for (int hf = 0; hf < 2; ++hf) {
@@ -231,12 +237,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             *reinterpret_cast<uint4*>(my_row + (((c32 * 4 + ch) ^ (row & 7)) << 4)) = pk;
           }
         }
-        fence_proxy_async();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (row == 0) {
-          tma_store_4d(&map_o, sm.o_stage, hf * 64, h, tl.r0, b);
-          bulk_commit();
-          stored = true;
+        if (rank) {
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          // thread t copies 16-byte chunk t & 7 of the staged rows (t >> 3) + 16 j to the rows' places
+          const int ch = row & 7;
+#pragma unroll 2
+          for (int j = 0; j < 8; ++j) {
+            const int r = (row >> 3) + 16 * j;
+            const int dst = tl.r0 + r < n ? rank[tl.r0 + r] : -1;
+            if (dst >= 0)
+              *reinterpret_cast<uint4*>(out_bh + (int64_t)dst * a.osn + hf * 64 + ch * 8) =
+                  *reinterpret_cast<const uint4*>(sm.o_stage + r * 128 + ((ch ^ (r & 7)) << 4));
+          }
+        } else {
+          fence_proxy_async();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (row == 0) {
+            tma_store_4d(&map_o, sm.o_stage, hf * 64, h, tl.r0, b);
+            bulk_commit();
+            stored = true;
+          }
         }
       }
       ring0 += nkt;
@@ -254,7 +274,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // Q of tile `it` goes into buffer it & 1 once the S MMAs of tile it - 2 have read it.
       auto load_q = [&](int it) {
         Tile tl;
-        if (!tile_at(it, part, parts, n, &tl)) return;
+        if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) return;
         const int bq = it & 1;
         if (it >= 2) ok = mbar_wait(&sm.q_empty[bq], ((it - 2) >> 1) & 1, abort_flag, a.status, code);
         if (!ok) return;
@@ -265,7 +285,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       load_q(0);
       for (int it = 0; ok; ++it) {
         Tile tl;
-        if (!tile_at(it, part, parts, n, &tl)) break;   // longest tile first
+        if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;   // longest tile first
         // Key tiles go up in even tiles of the walk and down in odd ones: the tiles read last are
         // the first ones the next tile reads, so they are still in L2.
         const bool down = it & 1;
@@ -295,7 +315,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int kv = 0;
       for (int it = 0; ok; ++it) {
         Tile tl;
-        if (!tile_at(it, part, parts, n, &tl)) break;
+        if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;
         const bool down = it & 1;
         for (int jj = 0; jj < tl.nkt && ok; ++jj, ++kv) {
           const int j = down ? tl.nkt - 1 - jj : jj;
@@ -319,7 +339,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int ring = 0;                                    // K tiles so far; buffer and stage ring & 1, phase (ring >> 1) & 1
       for (int it = 0; ok; ++it) {
         Tile tl;
-        if (!tile_at(it, part, parts, n, &tl)) break;
+        if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;
         const int bq = it & 1;
         ok = mbar_wait(&sm.q_full[bq], (it >> 1) & 1, abort_flag, a.status, code);
         const uint64_t dq = bq ? dq1 : dq0;
@@ -354,7 +374,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int ring = 0;
       for (int it = 0; ok; ++it) {
         Tile tl;
-        if (!tile_at(it, part, parts, n, &tl)) break;
+        if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;
         // the first PV of a tile overwrites the accumulator of the tile before it
         if (it >= 1) ok = mbar_wait(&sm.o_free, (it - 1) & 1, abort_flag, a.status, code);
         for (int j = 0; j < tl.nkt && ok; ++j, ++ring) {
@@ -391,7 +411,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     for (int it = 0; ok; ++it) {
       Tile tl;
-      if (!tile_at(it, part, parts, n, &tl)) break;
+      if (!tile_at(it, part, parts, n, a.tile_k0, a.tile_k1, &tl)) break;
       const int nkt = tl.nkt;
       const int i = tl.r0 + row;                          // query row of this thread
       const int tp = it & 1;
@@ -541,7 +561,9 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
   // One CTA per (sequence, head) when that fills the SMs evenly; otherwise deal each head's tiles
   // to 2, 4 or 8 CTAs. Cost model: waves of CTAs x the largest share of key-tile steps a CTA gets
   // (a tile costs about one step more, a CTA about two); splitting must win by 5 % to be chosen.
-  const int ntiles = (a.n + kTile - 1) / kTile;
+  const int all_tiles = (a.n + kTile - 1) / kTile;
+  const int ntiles = (a.tile_k1 < all_tiles ? a.tile_k1 : all_tiles) - a.tile_k0;    // tiles of this launch
+  if (ntiles <= 0) return cudaSuccess;
   const long long heads = (long long)a.Hq * a.B;
   int parts = 1;
   long long best = -1;
@@ -550,7 +572,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, cudaStream_t s) {
     for (int part = 0; part < p; ++part) {
       long long w = 0;
       Tile tl;
-      for (int it = 0; tile_at(it, part, p, a.n, &tl); ++it) w += tl.nkt + 1;
+      for (int it = 0; tile_at(it, part, p, a.n, a.tile_k0, a.tile_k1, &tl); ++it) w += tl.nkt + 1;
       if (w + 2 > share) share = w + 2;
     }
     const long long cost = ((heads * p + sms - 1) / sms) * share;

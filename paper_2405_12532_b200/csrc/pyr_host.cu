@@ -26,7 +26,7 @@ std::atomic<uint64_t> g_launches{0};   // kernels launched by this process throu
 std::atomic<int> g_sm_count[64];        // per device, 0 = not asked yet
 
 struct Layout {
-  size_t status, w, score, score_part, lse, idx, pos0, pos1, part_acc, part_ml, gen_part, total;
+  size_t status, w, score, score_part, lse, idx, rank, pos0, pos1, part_acc, part_ml, gen_part, total;
   int q_ring;            // rows of a layer's query ring (0: no generation-phase re-selection)
   std::vector<LayerPlan> layers;
 };
@@ -80,6 +80,8 @@ void plan(const pyr_config_t* c, Layout* lay) {
     off = align_up(off + B * Hq * (size_t)pyr::score_tc_chunks(L) * pyr::score_tc_groups() * (size_t)c0 * 4, kAlign);
   lay->lse = off;    off = align_up(off + B * Hq * (size_t)N * 4, kAlign);
   lay->idx = off;    off = align_up(off + B * G * (size_t)N * 4, kAlign);
+  lay->rank = off;
+  if (c->flags & PYR_FLAG_SELECT_FIRST) off = align_up(off + B * G * (size_t)N * 4, kAlign);   // the inverse of idx
   lay->pos0 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);
   lay->pos1 = off;   off = align_up(off + B * G * (size_t)N * 4, kAlign);
   lay->part_acc = off;
@@ -149,6 +151,9 @@ struct pyr_cache {
   int last_prefilled;
   bool needs_init;
   bool wait_test_armed;   // pyr_cache_arm_wait_test: the next decode call's loader leaves a chunk out
+  const void* sf_out;     // select-first ordering: the output tensor whose rows the last prefill wrote in kept order
+                          // (null: the selection has not run yet)
+  int sf_boundary;        // first row of the query tiles that were written before the selection
   float scale;
 };
 
@@ -241,6 +246,7 @@ pyr_status_t pyr_cache_alloc(const pyr_config_t* cfg, void* dev_buf, size_t byte
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
   c->needs_init = true;
   c->wait_test_armed = false;
+  c->sf_out = nullptr; c->sf_boundary = 0;
   c->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
   } catch (...) {           // the host-side vectors could not be allocated
     delete c;
@@ -259,6 +265,7 @@ pyr_status_t pyr_cache_free(pyr_cache_t* c) {
 pyr_status_t pyr_cache_reset(pyr_cache_t* c, void* stream) {
   if (!c) return PYR_ERR_NULL;
   c->next_layer = 0; c->phase = 0; c->pos_cur = 0; c->last_selected = -1; c->last_prefilled = -1;
+  c->sf_out = nullptr;
   std::fill(c->len_now.begin(), c->len_now.end(), 0);
   std::fill(c->q_count.begin(), c->q_count.end(), 0);
   return device_init(c, static_cast<cudaStream_t>(stream));
@@ -321,6 +328,23 @@ pyr_status_t pyr_cache_status(pyr_cache_t* c, void* stream, int32_t* host_status
   return word == 0 ? PYR_OK : PYR_ERR_TIMEOUT;
 }
 
+namespace {
+// the selection of layer `layer` as both orderings launch it (the position buffers swap when the layer is done)
+pyr::SelectArgs select_args(pyr_cache* c, int layer) {
+  const LayerPlan& p = c->lay.layers[layer];
+  int32_t* pos_in = at<int32_t>(c, c->pos_cur ? c->lay.pos1 : c->lay.pos0);
+  int32_t* pos_out = at<int32_t>(c, c->pos_cur ? c->lay.pos0 : c->lay.pos1);
+  pyr::SelectArgs sa;
+  sa.score = at<float>(c, c->lay.score);
+  sa.idx = at<int32_t>(c, c->lay.idx);
+  sa.pos_in = layer == 0 ? nullptr : pos_in;
+  sa.pos_out = pos_out;
+  sa.B = c->cfg.batch; sa.G = c->cfg.sel_groups; sa.n = p.n_in; sa.c = p.c; sa.k = p.k;
+  sa.reencode = (c->cfg.flags & PYR_FLAG_POS_REENCODE) ? 1 : 0;
+  return sa;
+}
+}  // namespace
+
 pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, const void* k, const void* v,
                                void* out, int64_t qsb, int64_t qsn, int64_t qsh, int64_t ksb, int64_t ksn,
                                int64_t ksh, int64_t osb, int64_t osn, int64_t osh, void* stream) {
@@ -354,13 +378,32 @@ pyr_status_t pyr_prefill_layer(pyr_cache_t* c, int32_t layer, const void* q, con
   const bool want_tc = c->cfg.dtype == PYR_BF16 && !(c->cfg.flags & PYR_FLAG_CUDA_CORE_PREFILL);
   const bool tc_attn = want_tc && pyr::prefill_tc_supported(a);
   const bool tc_score = want_tc && pyr::score_tc_supported(a);
-  cudaError_t e = tc_attn ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
-  if (e != cudaSuccess) return PYR_ERR_CUDA;
-  g_launches += 1;
-  if (p.c > 0) {
-    e = tc_score ? pyr::launch_score_tc(a, at<float>(c, c->lay.score_part), s) : pyr::launch_score_simt(a, s);
+  cudaError_t e;
+  c->sf_out = nullptr;
+  if ((c->cfg.flags & PYR_FLAG_SELECT_FIRST) && tc_attn && tc_score && p.c > 0 && p.k < p.c) {
+    // Select-first ordering: the query tiles that hold the window, the scores, the selection, and then the
+    // rest of the tiles, whose rows go straight to their places among the kept rows.
+    const int tiles = (p.n_in + 127) / 128, first_window_tile = p.c / 128;
+    a.tile_k0 = 0; a.tile_k1 = tiles - first_window_tile;
+    if (pyr::launch_prefill_tc(a, s) != cudaSuccess) return PYR_ERR_CUDA;
+    if (pyr::launch_score_tc(a, at<float>(c, c->lay.score_part), s) != cudaSuccess) return PYR_ERR_CUDA;
+    pyr::SelectArgs sa = select_args(c, layer);
+    sa.rank = at<int32_t>(c, c->lay.rank);
+    if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
+    a.tile_k0 = a.tile_k1; a.tile_k1 = 1 << 30; a.rank = sa.rank;
+    if (pyr::launch_prefill_tc(a, s) != cudaSuccess) return PYR_ERR_CUDA;
+    g_launches += first_window_tile > 0 ? 5 : 4;
+    c->sf_out = out;
+    c->sf_boundary = first_window_tile * 128;
+  } else {
+    e = tc_attn ? pyr::launch_prefill_tc(a, s) : pyr::launch_prefill_simt(a, s);
     if (e != cudaSuccess) return PYR_ERR_CUDA;
-    g_launches += tc_score ? 2 : 1;
+    g_launches += 1;
+    if (p.c > 0) {
+      e = tc_score ? pyr::launch_score_tc(a, at<float>(c, c->lay.score_part), s) : pyr::launch_score_simt(a, s);
+      if (e != cudaSuccess) return PYR_ERR_CUDA;
+      g_launches += tc_score ? 2 : 1;
+    }
   }
   if (c->lay.q_ring > 0) {
     // the window's queries go to the layer's ring: the generation phase re-scores the cache with them
@@ -401,17 +444,12 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const LayerPlan& p = c->lay.layers[layer];
-  int32_t* pos_in = at<int32_t>(c, c->pos_cur ? c->lay.pos1 : c->lay.pos0);
-  int32_t* pos_out = at<int32_t>(c, c->pos_cur ? c->lay.pos0 : c->lay.pos1);
-
-  pyr::SelectArgs sa;
-  sa.score = at<float>(c, c->lay.score);
-  sa.idx = at<int32_t>(c, c->lay.idx);
-  sa.pos_in = layer == 0 ? nullptr : pos_in;
-  sa.pos_out = pos_out;
-  sa.B = c->cfg.batch; sa.G = c->cfg.sel_groups; sa.n = p.n_in; sa.c = p.c; sa.k = p.k;
-  sa.reencode = (c->cfg.flags & PYR_FLAG_POS_REENCODE) ? 1 : 0;
-  if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
+  const pyr::SelectArgs sa = select_args(c, layer);
+  const bool selected = c->sf_out != nullptr;          // select-first ordering: the prefill call has run the selection
+  if (!selected) {
+    if (pyr::launch_select(sa, s) != cudaSuccess) return PYR_ERR_CUDA;
+    g_launches += 1;
+  }
 
   pyr::GatherArgs ga;
   ga.k = k; ga.v = v;
@@ -420,7 +458,7 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
   ga.B = c->cfg.batch; ga.Hkv = c->cfg.n_kv_heads; ga.G = c->cfg.sel_groups; ga.D = D;
   ga.n_out = p.n_out; ga.cap = p.cap; ga.elem_bytes = eb;
   if (pyr::launch_gather_kv(ga, s) != cudaSuccess) return PYR_ERR_CUDA;
-  g_launches += 2;
+  g_launches += 1;
 
   if (rows && p.n_out < p.n_in) {
     pyr::RowsArgs ra;
@@ -428,9 +466,16 @@ pyr_status_t pyr_select_compact(pyr_cache_t* c, int32_t layer, const void* k, co
     ra.row_elems = row_elems; ra.B = c->cfg.batch; ra.G = c->cfg.sel_groups; ra.n_out = p.n_out;
     ra.elem_bytes = eb;
     ra.idx_div = 1;
+    if (selected && rows == c->sf_out) {
+      // these are the rows the prefill call wrote: all but those of the tiles that held the window are in
+      // place; a row moves up by at most the number of rows dropped
+      ra.src_begin = c->sf_boundary;
+      ra.dst_begin = c->sf_boundary - (p.n_in - p.n_out) > 0 ? c->sf_boundary - (p.n_in - p.n_out) : 0;
+    }
     if (pyr::launch_compact_rows(ra, s) != cudaSuccess) return PYR_ERR_CUDA;
     g_launches += 1;
   }
+  c->sf_out = nullptr;
   if (n_out) *n_out = p.n_out;
   c->len_now[layer] = p.n_out;
   c->pos_cur ^= 1;

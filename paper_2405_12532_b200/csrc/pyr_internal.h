@@ -22,6 +22,11 @@ struct PrefillArgs {
   float scale;
   int dtype;
   int* status;
+  // select-first ordering (tcgen05 path): only the query tiles k0 <= k < k1, numbered from the last (longest) tile,
+  // are computed; with `rank` ([B, G, n]: a row's place among the kept rows of its selection group, -1 if dropped)
+  // every output row goes to its place instead of its own row
+  int tile_k0 = 0, tile_k1 = 1 << 30;
+  const int32_t* rank = nullptr;
 };
 
 struct SelectArgs {
@@ -31,6 +36,7 @@ struct SelectArgs {
   int32_t* pos_out;    // [B, G, n_out]
   int B, G, n, c, k;   // n_out = k + (n - c)
   int reencode = 0;    // 1: positions are re-encoded from 0 in kept order instead of gathered
+  int32_t* rank = nullptr;   // [B, G, n] or nullptr: the inverse of idx (-1 for dropped rows)
 };
 
 struct GatherArgs {
@@ -47,6 +53,8 @@ struct RowsArgs {
   int64_t row_elems;
   int B, G, n_out, elem_bytes;
   int idx_div;         // consecutive row groups that share one index list (1: a list per group)
+  int dst_begin = 0;   // rows below this destination, and rows whose source lies below src_begin, are in place already
+  int src_begin = 0;
 };
 
 // Generation-phase score of a layer's cache from its window of recent queries.

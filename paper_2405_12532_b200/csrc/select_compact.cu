@@ -35,17 +35,23 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
   int32_t* idx = a.idx + (int64_t)bg * n_out;
   int32_t* pos_out = a.pos_out + (int64_t)bg * n_out;
   const int32_t* pos_in = a.pos_in ? a.pos_in + (int64_t)bg * n : nullptr;
+  int32_t* rank = a.rank ? a.rank + (int64_t)bg * n : nullptr;
 
   // the window is always kept
   for (int i = t; i < window; i += kSelThreads) {
     idx[k + i] = c + i;
     pos_out[k + i] = a.reencode ? k + i : (pos_in ? pos_in[c + i] : c + i);
+    if (rank) rank[c + i] = k + i;
   }
-  if (k == 0) return;
+  if (k == 0) {
+    if (rank) for (int i = t; i < c; i += kSelThreads) rank[i] = -1;
+    return;
+  }
   if (k == c) {
     for (int i = t; i < c; i += kSelThreads) {
       idx[i] = i;
       pos_out[i] = a.reencode ? i : (pos_in ? pos_in[i] : i);
+      if (rank) rank[i] = i;
     }
     return;
   }
@@ -123,6 +129,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a) {
       const uint32_t p = gt_before + min(eq_before, need_eq);
       idx[p] = i;
       pos_out[p] = a.reencode ? (int)p : (pos_in ? pos_in[i] : i);
+      if (rank) rank[i] = (int)p;
+    } else if (rank && i < c) {
+      rank[i] = -1;
     }
     __syncthreads();
     if (t == kSelThreads - 1) sh_running = before + (gt ? (1u << 16) : 0u) + (eq ? 1u : 0u);
@@ -207,7 +216,7 @@ __global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, i
       dr[u] = -1;
       if (rr < rows_per_iter && r0 + rr < a.n_out) {
         const int src = idx[r0 + rr];
-        if (src != r0 + rr) {             // rows already in place are not touched
+        if (src != r0 + rr && src >= a.src_begin) {   // rows already in place are not touched
           dr[u] = r0 + rr;
           bf[u] = *reinterpret_cast<const uint4*>(base + (int64_t)src * row_bytes + ln[u] * 16);
         }
@@ -219,9 +228,10 @@ __global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, i
     for (int u = 0; u < kRowUnroll; ++u)
       if (dr[u] >= 0) *reinterpret_cast<uint4*>(base + (int64_t)dr[u] * row_bytes + ln[u] * 16) = bf[u];
   };
-  read_chunk(0, buf[0], dst_row[0]);
+  const int first = a.dst_begin / rows_per_iter * rows_per_iter;
+  read_chunk(first, buf[0], dst_row[0]);
   __syncthreads();
-  for (int r0 = 0; r0 < a.n_out; r0 += 2 * rows_per_iter) {
+  for (int r0 = first; r0 < a.n_out; r0 += 2 * rows_per_iter) {
     if (r0 + rows_per_iter < a.n_out) read_chunk(r0 + rows_per_iter, buf[1], dst_row[1]);
     write_chunk(buf[0], dst_row[0]);
     __syncthreads();

@@ -213,6 +213,36 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (i < n) a.lse[((int64_t)b * a.Hq + h) * n + i] = (m_fin + log2f(l)) * kLn2;
       const float inv = 1.f / l;
 
+      if (rank) {
+        // The row goes to its place among the kept rows, straight from registers: a thread writes whole
+        // 128-byte lines of its own row, 16 columns of the accumulator at a time (the epilogue warps are
+        // short of registers), and the accumulator is free for the next tile after the last load.
+        const int dst = i < n ? rank[i] : -1;
+        __nv_bfloat16* orow = out_bh + (int64_t)(dst >= 0 ? dst : 0) * a.osn;
+#pragma unroll
+        for (int c16 = 0; c16 < 8; ++c16) {
+          uint32_t o[16];
+          tmem_ld16(o_addr + c16 * 16, o);
+          tmem_wait_ld();
+          if (c16 == 7) {
+            tc_fence_before();
+            mbar_arrive(&sm.o_free);
+          }
+          if (dst >= 0) {
+            uint4 lo, hi;
+            lo.x = pack_bf16(__uint_as_float(o[0]) * inv, __uint_as_float(o[1]) * inv);
+            lo.y = pack_bf16(__uint_as_float(o[2]) * inv, __uint_as_float(o[3]) * inv);
+            lo.z = pack_bf16(__uint_as_float(o[4]) * inv, __uint_as_float(o[5]) * inv);
+            lo.w = pack_bf16(__uint_as_float(o[6]) * inv, __uint_as_float(o[7]) * inv);
+            hi.x = pack_bf16(__uint_as_float(o[8]) * inv, __uint_as_float(o[9]) * inv);
+            hi.y = pack_bf16(__uint_as_float(o[10]) * inv, __uint_as_float(o[11]) * inv);
+            hi.z = pack_bf16(__uint_as_float(o[12]) * inv, __uint_as_float(o[13]) * inv);
+            hi.w = pack_bf16(__uint_as_float(o[14]) * inv, __uint_as_float(o[15]) * inv);
+            *reinterpret_cast<uint4*>(orow + c16 * 16) = lo;
+            *reinterpret_cast<uint4*>(orow + c16 * 16 + 8) = hi;
+          }
+        }
+      } else {
       // O leaves through shared memory, one [128 x 64] half at a time (rows past n are clipped by the store)
 #pragma unroll 1
       for (int hf = 0; hf < 2; ++hf) {
@@ -237,27 +267,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             *reinterpret_cast<uint4*>(my_row + (((c32 * 4 + ch) ^ (row & 7)) << 4)) = pk;
           }
         }
-        if (rank) {
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          // thread t copies 16-byte chunk t & 7 of the staged rows (t >> 3) + 16 j to the rows' places
-          const int ch = row & 7;
-#pragma unroll 2
-          for (int j = 0; j < 8; ++j) {
-            const int r = (row >> 3) + 16 * j;
-            const int dst = tl.r0 + r < n ? rank[tl.r0 + r] : -1;
-            if (dst >= 0)
-              *reinterpret_cast<uint4*>(out_bh + (int64_t)dst * a.osn + hf * 64 + ch * 8) =
-                  *reinterpret_cast<const uint4*>(sm.o_stage + r * 128 + ((ch ^ (r & 7)) << 4));
-          }
-        } else {
-          fence_proxy_async();
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (row == 0) {
-            tma_store_4d(&map_o, sm.o_stage, hf * 64, h, tl.r0, b);
-            bulk_commit();
-            stored = true;
-          }
+        fence_proxy_async();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (row == 0) {
+          tma_store_4d(&map_o, sm.o_stage, hf * 64, h, tl.r0, b);
+          bulk_commit();
+          stored = true;
         }
+      }
       }
       ring0 += nkt;
     }

@@ -126,7 +126,7 @@ class Workload:
     """Device-resident synthetic inputs and the call sequence of one step."""
 
     def __init__(self, name: str, device, pool: int = 2, layers: int = 0, decode_steps: int = -1, batch: int = 0,
-                 reselect_every: int = 0, select_first: bool = False):
+                 reselect_every: int = 0, select_first: str = "auto"):
         from paper_2405_12532_b200 import binding as pb
         self.pb = pb
         self.name = name
@@ -142,10 +142,12 @@ class Workload:
             w["batch"] = batch
         self.reselect_every = reselect_every      # generation-phase PvC update every so many decode steps (0: never)
         flags = pb.PYR_FLAG_GEN_RESELECT if reselect_every else 0
-        # Select-first ordering (on request) where the rows that select + compact moves are the attention output itself
-        # (one kept set per head group): the kept rows are then written in place by the attention kernel. With one
-        # kept set per sequence the compacted rows are the hidden states, which attention does not produce.
-        self.select_first = bool(select_first and w["sel_groups"] > 1 and w["dtype"] == "bf16" and w["head_dim"] == 128)
+        # Select-first ordering where the rows that select + compact moves are the attention output itself (one kept
+        # set per head group): the kept rows are then written in place by the attention kernel. With one kept set per
+        # sequence the compacted rows are the hidden states, which attention does not produce. "auto": on for prompts
+        # of 4096 tokens and more, where it was measured to win (its two attention launches cost more on short ones).
+        want = select_first == "on" or (select_first == "auto" and w["prompt_len"] >= 4096)
+        self.select_first = bool(want and w["sel_groups"] > 1 and w["dtype"] == "bf16" and w["head_dim"] == 128)
         if self.select_first:
             flags |= pb.PYR_FLAG_SELECT_FIRST
         self.cache = pb.PyrCache(device=device, **pb.config_from_workload(w, self.ratio, flags=flags))
@@ -768,9 +770,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--select-first", action="store_true",
+    ap.add_argument("--select-first", default="auto", choices=["auto", "on", "off"],
                     help="select-first ordering on the per-head workloads: the window's query tiles, the scores and the "
-                         "selection first, then the other tiles writing kept rows in place")
+                         "selection first, then the other tiles writing kept rows in place (auto: prompts of 4096 tokens and more)")
     ap.add_argument("--no-model", action="store_true", help="skip the whole-model run that the default workload reports beside its line")
     ap.add_argument("--reselect-every", type=int, default=0,
                     help="generation-phase PvC update of every layer every so many decode steps (0: never)")

@@ -209,3 +209,13 @@ def test_glue_entry_points_validate_before_any_launch():
     assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(2), i32(0), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_INVALID
     assert L.pyr_glue_linear_rows(P, P, NULL, P, i64(4), P, i32(2), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_NULL
     assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(0), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_OK
+
+
+def test_select_first_flag_adds_the_inverse_list_to_the_plan():
+    """PYR_FLAG_SELECT_FIRST carves one more [B, G, N] int32 array (the inverse of the kept list), nothing else."""
+    base_cfg, keep0 = _cfg()
+    flag_cfg, keep1 = _cfg(flags=pb.PYR_FLAG_SELECT_FIRST)
+    b0, _ = pb.pyr_cache_bytes(base_cfg)
+    b1, _ = pb.pyr_cache_bytes(flag_cfg)
+    want = 2 * 4 * 512 * 4                     # B * G * N * 4 bytes
+    assert b1 - b0 == (want + 255) // 256 * 256

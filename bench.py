@@ -301,8 +301,14 @@ class ModelWorkload(Workload):
         rn = lambda *s: (torch.randn(*s, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
         self.W = {"emb": rn(V, d), "head": rn(V, d), "nf": torch.ones(d, device=device, dtype=torch.bfloat16)}
         for l in range(w["n_layers"]):
-            for nm, shape in (("wq", (d, d)), ("wk", (d, d)), ("wv", (d, d)), ("wo", (d, d)), ("wg", (f, d)), ("wu", (f, d)), ("wd", (d, f))):
-                self.W[f"{nm}{l}"] = rn(*shape)
+            # q, k, v and gate, up are stored stacked: a decode step streams each stack through one launch, the
+            # prefill uses the row blocks as separate weights
+            self.W[f"wqkv{l}"] = rn(3 * d, d)
+            self.W[f"wgu{l}"] = rn(2 * f, d)
+            for i, nm in enumerate(("wq", "wk", "wv")):
+                self.W[f"{nm}{l}"] = self.W[f"wqkv{l}"][i * d:(i + 1) * d]
+            self.W[f"wg{l}"], self.W[f"wu{l}"] = self.W[f"wgu{l}"][:f], self.W[f"wgu{l}"][f:]
+            self.W[f"wo{l}"], self.W[f"wd{l}"] = rn(d, d), rn(d, f)
             self.W[f"n1{l}"] = torch.ones(d, device=device, dtype=torch.bfloat16)
             self.W[f"n2{l}"] = torch.ones(d, device=device, dtype=torch.bfloat16)
         self.ids = synth.uniform_token_ids(B, N, V, seed=0).to(torch.int32).to(device)
@@ -350,14 +356,14 @@ class ModelWorkload(Workload):
             p = torch.full((B,), N + t, device=self.device, dtype=torch.int32)
             for l in range(w["n_layers"]):
                 h = pb.glue_rmsnorm(xt, W[f"n1{l}"])
-                q = pb.glue_rope_(pb.glue_linear(h, W[f"wq{l}"]).view(B, H, D), p)
-                k = pb.glue_rope_(pb.glue_linear(h, W[f"wk{l}"]).view(B, H, D), p)
-                v = pb.glue_linear(h, W[f"wv{l}"]).view(B, H, D)
+                q, k, v = pb.glue_linear_split(h, W[f"wqkv{l}"], 3)
+                q, k, v = pb.glue_rope_(q.view(B, H, D), p), pb.glue_rope_(k.view(B, H, D), p), v.view(B, H, D)
                 o = torch.empty_like(q)
                 c.decode_attn(l, q, k, v, o)
                 y = pb.glue_linear(o.view(B, d), W[f"wo{l}"], xt)
                 h2 = pb.glue_rmsnorm(y, W[f"n2{l}"])
-                xt = pb.glue_linear(pb.glue_swiglu(pb.glue_linear(h2, W[f"wg{l}"]), pb.glue_linear(h2, W[f"wu{l}"])), W[f"wd{l}"], y)
+                g, u = pb.glue_linear_split(h2, W[f"wgu{l}"], 2)
+                xt = pb.glue_linear(pb.glue_swiglu(g, u), W[f"wd{l}"], y)
             self.last_token = pb.glue_argmax(pb.glue_linear(pb.glue_rmsnorm(xt, W["nf"]), W["head"]))
             if self.reselect_every and (t + 1) % self.reselect_every == 0:
                 for l in range(w["n_layers"]):

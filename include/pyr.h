@@ -340,6 +340,10 @@ pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
  *           rows_stride + i], :] for x [batch, n_dst, k], residual [batch, n_src, n], y [batch, n_dst, n].
  *           The lists are device int32 (pyr_cache_kept's first pointer, a dense [B, n_out] array when
  *           sel_groups == 1: rows_stride = n_out); their entries must lie in [0, n_src), which is not checked.
+ *   linear_split  the product of x [m, k] with a weight [n_parts * part_n, k] of up to four stacked
+ *           projections (say q, k and v), part i written to its own tensor ys[i] [m, part_n] (ys: host
+ *           array of device pointers): for at most 64 rows of x in bf16 the weight streams through one
+ *           launch instead of one per projection; otherwise it is one product per part.
  *   linear_swiglu  out[m, n] = silu(x . w_gate^T) * (x . w_up^T), w_gate and w_up [n, k]: the gated MLP's
  *           first half in one pass, neither projection written out (fp32 accumulators go straight
  *           into the product). bf16 with 16-byte aligned pointers, k a multiple of 64 and n a
@@ -363,6 +367,8 @@ pyr_status_t pyr_glue_rmsnorm_rows(const void* x, const int32_t* rows, int64_t r
 pyr_status_t pyr_glue_linear_rows(const void* x, const void* w, const void* residual, const int32_t* res_rows,
                                   int64_t rows_stride, void* y, int32_t batch, int32_t n_src, int32_t n_dst, int32_t n,
                                   int32_t k, int32_t dtype, void* stream);
+pyr_status_t pyr_glue_linear_split(const void* x, const void* w, void* const* ys, int32_t n_parts, int64_t m, int32_t part_n,
+                                   int32_t k, int32_t dtype, void* stream);
 pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
                                     int32_t k, int32_t dtype, void* stream);
 pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,

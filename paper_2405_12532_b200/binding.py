@@ -26,7 +26,7 @@ PYR_FLAG_SELECT_FIRST = 8
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_swiglu", "pyr_glue_rmsnorm_rows", "pyr_glue_linear_rows",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_split", "pyr_glue_linear_swiglu", "pyr_glue_rmsnorm_rows", "pyr_glue_linear_rows",
     "pyr_glue_rope", "pyr_glue_swiglu", "pyr_glue_argmax", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
         L.pyr_glue_rmsnorm.argtypes = [vp, vp, vp, i64, i32, C.c_float, i32, vp]
         L.pyr_glue_linear.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
         L.pyr_glue_linear_swiglu.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp]
+        L.pyr_glue_linear_split.argtypes = [vp, vp, vp, i32, i64, i32, i32, i32, vp]
         L.pyr_glue_rmsnorm_rows.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, C.c_float, i32, vp]
         L.pyr_glue_linear_rows.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i32, i32, i32, i32, vp]
         L.pyr_glue_rope.argtypes = [vp, vp, i64, i32, i32, i32, vp]
@@ -223,6 +224,18 @@ def glue_linear_rows(x, w, residual, res_rows):
                                       y.data_ptr(), B, residual.shape[1], n_dst, N, K, _dt(x), C.c_void_p(_stream_ptr(None))),
            "pyr_glue_linear_rows")
     return y
+
+
+def glue_linear_split(x, w, n_parts: int):
+    """x [..., K] . w [n_parts * part_n, K]^T as n_parts tensors [..., part_n] (pyr_glue_linear_split)."""
+    assert x.is_contiguous() and w.is_contiguous() and w.shape[0] % n_parts == 0
+    K = w.shape[1]
+    part_n = w.shape[0] // n_parts
+    ys = [torch.empty(*x.shape[:-1], part_n, dtype=x.dtype, device=x.device) for _ in range(n_parts)]
+    arr = (C.c_void_p * n_parts)(*[y.data_ptr() for y in ys])
+    _check(lib().pyr_glue_linear_split(x.data_ptr(), w.data_ptr(), arr, n_parts, x.numel() // K, part_n, K, _dt(x),
+                                       C.c_void_p(_stream_ptr(None))), "pyr_glue_linear_split")
+    return ys
 
 
 def glue_linear_swiglu(x, w_gate, w_up):

@@ -43,9 +43,12 @@ struct SkSmem {
 static_assert(kSkM * kRedStride * 4 <= kSkStages * kSkWBytes, "partial sums reuse the weight ring");
 static_assert(2 * (sizeof(SkSmem) + 1024 + 1024) <= 228 * 1024, "two CTAs per SM");
 
+constexpr int kSkMaxParts = 4;
+
 struct SkinnyArgs {
   const __nv_bfloat16* res;
-  __nv_bfloat16* y;
+  __nv_bfloat16* y[kSkMaxParts];   // the output's column parts, each [M, part_n] (one part: the whole of y)
+  int part_n;
   int M, N, K, ktiles;      // ktiles = [64-wide] K tiles in all; slice i takes [i ktiles / slices, (i + 1) ktiles / slices)
   int* status;              // may be null
 };
@@ -168,7 +171,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       } else {
         v = *reinterpret_cast<const float4*>(&red[r * kRedStride + c4]);
       }
-      const int64_t o = (int64_t)r * a.N + n0 + c4;
+      const int part = n0 / a.part_n;                        // a feature block lies within one part (part_n % 128 == 0)
+      const int64_t o = (int64_t)r * a.part_n + (n0 - part * a.part_n) + c4;
       if (a.res) {
         const uint2 rr = *reinterpret_cast<const uint2*>(a.res + o);
         v.x += __uint_as_float(rr.x << 16); v.y += __uint_as_float(rr.x & 0xffff0000u);
@@ -177,7 +181,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       uint2 ov;
       ov.x = pack_bf16(v.x, v.y);
       ov.y = pack_bf16(v.z, v.w);
-      *reinterpret_cast<uint2*>(a.y + o) = ov;
+      *reinterpret_cast<uint2*>(a.y[part] + o) = ov;
     }
   }
   if (slices > 1) cluster_sync_all(); else __syncthreads();     // peers may still be reading this CTA's partial sums
@@ -205,8 +209,10 @@ bool gemm_skinny_supported(const void* x, const void* w, const void* res, const 
   return tensor_maps_available() && al % 16 == 0 && M >= 1 && M <= kSkM && N % kSkN == 0 && K % kSkK == 0;
 }
 
-cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
-                               cudaStream_t s) {
+cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* const* ys, int n_parts, int64_t M, int N,
+                               int K, int* status, cudaStream_t s) {
+  if (n_parts < 1 || n_parts > kSkMaxParts || N % n_parts || (n_parts > 1 && ((N / n_parts) % kSkN || res)))
+    return cudaErrorInvalidValue;
   const int sms = device_sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   const int smem = (int)sizeof(SkSmem) + 1024;
@@ -218,7 +224,9 @@ cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, vo
     return cudaErrorInvalidValue;
   const int slices = skinny_slices(N, K, sms);
   SkinnyArgs a;
-  a.res = static_cast<const __nv_bfloat16*>(res); a.y = static_cast<__nv_bfloat16*>(y);
+  a.res = static_cast<const __nv_bfloat16*>(res);
+  for (int i = 0; i < kSkMaxParts; ++i) a.y[i] = static_cast<__nv_bfloat16*>(ys[i < n_parts ? i : 0]);
+  a.part_n = N / n_parts;
   a.M = (int)M; a.N = N; a.K = K; a.ktiles = K / kSkK; a.status = status;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(N / kSkN, slices, 1);

@@ -575,10 +575,34 @@ pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual,
   if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
   if (m == 0) return PYR_OK;
   if (dtype == PYR_BF16 && pyr::gemm_skinny_supported(x, w, residual, y, m, n, k))
-    PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, y, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
+    PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, &y, 1, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
   if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
     PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
   PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_linear_split(const void* x, const void* w, void* const* ys, int32_t n_parts, int64_t m, int32_t part_n,
+                                   int32_t k, int32_t dtype, void* stream) {
+  if (!ys) return PYR_ERR_NULL;
+  if (n_parts < 1 || n_parts > 4) return PYR_ERR_INVALID;
+  for (int i = 0; i < n_parts; ++i)
+    if (!ys[i]) return PYR_ERR_NULL;
+  if (!glue_ok(dtype, {x, w})) return dtype == PYR_BF16 || dtype == PYR_F32 ? PYR_ERR_NULL : PYR_ERR_UNSUPPORTED;
+  if (m < 0 || part_n < 1 || k < 1) return PYR_ERR_INVALID;
+  if (m == 0) return PYR_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int n = part_n * n_parts;
+  bool aligned = true;
+  for (int i = 0; i < n_parts; ++i) aligned = aligned && reinterpret_cast<uintptr_t>(ys[i]) % 16 == 0;
+  if (dtype == PYR_BF16 && aligned && part_n % 128 == 0 && pyr::gemm_skinny_supported(x, w, nullptr, ys[0], m, n, k))
+    PYR_GLUE(pyr::launch_gemm_skinny(x, w, nullptr, ys, n_parts, m, n, k, nullptr, s));
+  // otherwise one product per part, on the rows of w that belong to it
+  const size_t eb = dtype == PYR_BF16 ? 2 : 4;
+  for (int i = 0; i < n_parts; ++i) {
+    const pyr_status_t st = pyr_glue_linear(x, static_cast<const char*>(w) + (size_t)i * part_n * k * eb, nullptr, ys[i], m, part_n, k,
+                                            dtype, stream);
+    if (st != PYR_OK) return st;
+  }
+  return PYR_OK;
 }
 pyr_status_t pyr_glue_linear_rows(const void* x, const void* w, const void* residual, const int32_t* res_rows,
                                   int64_t rows_stride, void* y, int32_t batch, int32_t n_src, int32_t n_dst, int32_t n,

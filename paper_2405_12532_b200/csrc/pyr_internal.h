@@ -146,8 +146,9 @@ cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* 
 cudaError_t launch_gemm_tc_gated(const void* x, const void* wg, const void* wu, void* out, int64_t M, int N, int K,
                                  int* status, cudaStream_t s);
 bool gemm_skinny_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
-cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* y, int64_t M, int N, int K, int* status,
-                               cudaStream_t s);
+// y may be given as up to four column parts ys[i] of [M, N / n_parts] each (n_parts > 1: no residual, parts of whole 128s)
+cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* const* ys, int n_parts, int64_t M, int N,
+                               int K, int* status, cudaStream_t s);
 cudaError_t launch_glue_rope(void* x, const int32_t* pos, int64_t tokens, int H, int D, int dtype, cudaStream_t s);
 cudaError_t launch_glue_swiglu(const void* g, const void* u, void* out, int64_t n, int dtype, cudaStream_t s);
 cudaError_t launch_glue_argmax(const void* x, int32_t* out, int64_t rows, int n, int dtype, cudaStream_t s);

@@ -151,3 +151,22 @@ def test_row_mapped_norm_and_residual(dtype, tol):
         r2 = _r(B2, s2, 1024, seed=58, dtype=dtype)
         r2g = torch.gather(r2, 1, rows2.long()[:, :, None].expand(B2, d2, 1024)).contiguous()
         assert torch.equal(pb.glue_linear_rows(h2, w2, r2, rows2), pb.glue_linear(h2, w2, r2g))
+
+
+@pytest.mark.parametrize("M,parts,part_n,K", [(64, 3, 4096, 4096), (9, 2, 11008, 4096), (64, 4, 128, 192), (200, 3, 256, 128),
+                                              (7, 2, 100, 64)])
+def test_split_linear_equals_separate_products(M, parts, part_n, K):
+    """pyr_glue_linear_split: stacked projections through one weight-streaming launch (few rows, parts of whole
+    128s) or one product per part otherwise; either way each part equals x . w_part^T to bf16 rounding."""
+    x = _r(M, K, seed=61, dtype=torch.bfloat16)
+    w = (_r(parts * part_n, K, seed=62) * 0.05).to(torch.bfloat16)
+    launches = pb.launch_count()
+    ys = pb.glue_linear_split(x, w, parts)
+    torch.cuda.synchronize()
+    one_launch = M <= 64 and part_n % 128 == 0 and K % 64 == 0
+    assert pb.launch_count() - launches == (1 if one_launch else parts)
+    for i, y in enumerate(ys):
+        want = x.double() @ w[i * part_n:(i + 1) * part_n].double().T
+        scale = float(want.abs().max().clamp_min(1e-3))
+        assert y.shape == (M, part_n)
+        assert float((y.double() - want).abs().max()) <= 2 ** -7 * scale

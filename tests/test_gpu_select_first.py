@@ -107,3 +107,46 @@ def test_select_first_over_a_chain_of_layers_with_other_rows():
     torch.cuda.synchronize()
     assert cache.status() == 0
     cache.close()
+
+
+def test_select_first_with_reencoded_positions_and_generation_update():
+    """The flag combined with re-encoded positions and the generation-phase update: same kept lists, positions and
+    caches as the default ordering, before and after a re-selection during decode."""
+    Hq, Hkv, B, N, L, D, T = 4, 2, 2, 900, 128, 128, 6
+    w = dict(n_layers=2, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, sel_groups=Hkv, dtype="bf16", batch=B,
+             prompt_len=N, recent_len=L, max_new_tokens=T, hitter_frac=0.05, hitter_mag=3.0)
+    ratio = [0.8, 0.5]
+    base = pb.PYR_FLAG_POS_REENCODE | pb.PYR_FLAG_GEN_RESELECT
+    got = []
+    for flags in (base | pb.PYR_FLAG_SELECT_FIRST, base):
+        cache = pb.PyrCache(device=DEV, **pb.config_from_workload(w, ratio, flags=flags))
+        snap = []
+        for l in range(2):
+            n = cache.layer_info(l)["n_in"]
+            Q, K, V = synth.stack_layer_inputs(w, 30 + l, n, device=DEV, boost_queries=True)
+            out = torch.empty(B, n, Hq, D, device=DEV, dtype=torch.bfloat16)
+            cache.prefill_layer(l, Q, K, V, out)
+            per = Hq // Hkv
+            n_out = cache.select_compact(l, K, V, out, per * D, n * Hq * D, Hq * D, per * D)
+            kept, pos = cache.kept(l)
+            snap.append((kept.clone(), pos.clone(), n_out))
+        for t in range(4):
+            q, kn, vn = synth.decode_step_inputs(w, 0, t, device=DEV)
+            o = torch.empty_like(q)
+            for l in range(2):
+                cache.decode_attn(l, q, kn, vn, o)
+        for l in range(2):
+            cache.decode_reselect(l)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        caches = []
+        for l in range(2):
+            Kc, Vc = cache.kv(l)
+            ln = cache.layer_info(l)["len_now"]
+            caches.append((Kc[:, :, :ln].clone(), Vc[:, :, :ln].clone()))
+        got.append((snap, caches))
+        cache.close()
+    (s1, c1), (s0, c0) = got
+    for l in range(2):
+        assert torch.equal(s1[l][0], s0[l][0]) and torch.equal(s1[l][1], s0[l][1]) and s1[l][2] == s0[l][2]
+        assert torch.equal(c1[l][0], c0[l][0]) and torch.equal(c1[l][1], c0[l][1])

@@ -412,7 +412,7 @@ def run_model(args, rank, world, local_rank, name, emit=True):
     pdist.barrier(world)
     launches = pb.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    assert wl.cache.status() == 0
+    assert wl.cache.status() == 0 and pb.glue_status() == 0, "device-side wait timed out"
     t_pre = sum(m[0].elapsed_time(m[1]) for m in marks) / 1e3
     t_dec = sum(m[1].elapsed_time(m[2]) for m in marks) / 1e3
     t_pre, t_dec = pdist.max_over_ranks([t_pre, t_dec], world, device)

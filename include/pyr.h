@@ -355,6 +355,14 @@ pyr_status_t pyr_decode_attn_noalloc_status(void* stream, int32_t* host_status);
  *   swiglu  out = silu(gate) * up, n elements.
  *   argmax  out[r] = index of the largest of x[r, 0..n), the lowest index on ties; x [rows, n].
  */
+/*
+ * The tensor-core linear layers wait on their copies with bounded waits; a wait that runs out is
+ * recorded in a status word the library keeps per GPU (the glue calls have no cache handle).
+ * pyr_glue_status synchronises `stream` and reports 0 or PYR_ERR_TIMEOUT for the current GPU since the
+ * last report (reading clears the record); after a timeout the outputs of the calls since then are
+ * undefined. Allocates nothing.
+ */
+pyr_status_t pyr_glue_status(void* stream, int32_t* host_status);
 pyr_status_t pyr_glue_embed(const int32_t* ids, const void* table, void* out, int64_t tokens, int32_t d, int32_t vocab,
                             int32_t dtype, int32_t* dev_status, void* stream);
 pyr_status_t pyr_glue_rmsnorm(const void* x, const void* gain, void* out, int64_t tokens, int32_t d, float eps,

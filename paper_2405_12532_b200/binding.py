@@ -26,7 +26,7 @@ PYR_FLAG_SELECT_FIRST = 8
 EXPORTS = [
     "pyr_cache_layer_info", "pyr_cache_bytes", "pyr_cache_alloc", "pyr_cache_free", "pyr_cache_reset",
     "pyr_cache_kept", "pyr_cache_scores", "pyr_cache_lse", "pyr_cache_kv", "pyr_cache_status",
-    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_linear", "pyr_glue_linear_split", "pyr_glue_linear_swiglu", "pyr_glue_rmsnorm_rows", "pyr_glue_linear_rows",
+    "pyr_prefill_layer", "pyr_select_compact", "pyr_decode_attn", "pyr_decode_reselect", "pyr_cache_arm_wait_test", "pyr_recent_len_from_ratio", "pyr_glue_embed", "pyr_glue_rmsnorm", "pyr_glue_status", "pyr_glue_linear", "pyr_glue_linear_split", "pyr_glue_linear_swiglu", "pyr_glue_rmsnorm_rows", "pyr_glue_linear_rows",
     "pyr_glue_rope", "pyr_glue_swiglu", "pyr_glue_argmax", "pyr_status_string", "pyr_version", "pyr_launch_count",
     "pyr_decode_attn_noalloc", "pyr_decode_attn_noalloc_status",
 ]
@@ -236,6 +236,13 @@ def glue_linear_split(x, w, n_parts: int):
     _check(lib().pyr_glue_linear_split(x.data_ptr(), w.data_ptr(), arr, n_parts, x.numel() // K, part_n, K, _dt(x),
                                        C.c_void_p(_stream_ptr(None))), "pyr_glue_linear_split")
     return ys
+
+
+def glue_status() -> int:
+    """0, or PYR_ERR_TIMEOUT if a linear layer's bounded wait ran out on this GPU since the last call (pyr_glue_status)."""
+    word = C.c_int32(0)
+    lib().pyr_glue_status(C.c_void_p(_stream_ptr(None)), C.byref(word))
+    return int(word.value)
 
 
 def glue_linear_swiglu(x, w_gate, w_up):

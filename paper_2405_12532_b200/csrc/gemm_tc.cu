@@ -18,6 +18,8 @@
 #include <cuda_bf16.h>
 #include <stddef.h>
 
+#include <mutex>
+
 #include "pyr_internal.h"
 #include "tc_common.cuh"
 
@@ -235,7 +237,26 @@ cudaError_t run_gemm(const CUtensorMap& mx, const CUtensorMap& mw, const CUtenso
   return cudaGetLastError();
 }
 
+// The glue calls have no cache handle, so the GEMMs' bounded waits report to a word of the library's own, one
+// per GPU (a static device variable: nothing is allocated).
+__device__ int g_glue_status = 0;
+constexpr int kGlueMaxDevices = 64;
+int* g_glue_status_ptr[kGlueMaxDevices] = {};
+std::mutex g_glue_mutex;
+
 }  // namespace
+
+int* glue_status_word() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kGlueMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_glue_mutex);
+  if (!g_glue_status_ptr[dev]) {
+    int* w = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&w), g_glue_status) != cudaSuccess) return nullptr;
+    g_glue_status_ptr[dev] = w;
+  }
+  return g_glue_status_ptr[dev];
+}
 
 bool gemm_tc_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K) {
   const uintptr_t al = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(y) |

@@ -575,9 +575,9 @@ pyr_status_t pyr_glue_linear(const void* x, const void* w, const void* residual,
   if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
   if (m == 0) return PYR_OK;
   if (dtype == PYR_BF16 && pyr::gemm_skinny_supported(x, w, residual, y, m, n, k))
-    PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, &y, 1, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
+    PYR_GLUE(pyr::launch_gemm_skinny(x, w, residual, &y, 1, m, n, k, pyr::glue_status_word(), static_cast<cudaStream_t>(stream)));
   if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
-    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
+    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, pyr::glue_status_word(), pyr::RowMap(), static_cast<cudaStream_t>(stream)));
   PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, pyr::RowMap(), static_cast<cudaStream_t>(stream)));
 }
 pyr_status_t pyr_glue_linear_split(const void* x, const void* w, void* const* ys, int32_t n_parts, int64_t m, int32_t part_n,
@@ -594,7 +594,7 @@ pyr_status_t pyr_glue_linear_split(const void* x, const void* w, void* const* ys
   bool aligned = true;
   for (int i = 0; i < n_parts; ++i) aligned = aligned && reinterpret_cast<uintptr_t>(ys[i]) % 16 == 0;
   if (dtype == PYR_BF16 && aligned && part_n % 128 == 0 && pyr::gemm_skinny_supported(x, w, nullptr, ys[0], m, n, k))
-    PYR_GLUE(pyr::launch_gemm_skinny(x, w, nullptr, ys, n_parts, m, n, k, nullptr, s));
+    PYR_GLUE(pyr::launch_gemm_skinny(x, w, nullptr, ys, n_parts, m, n, k, pyr::glue_status_word(), s));
   // otherwise one product per part, on the rows of w that belong to it
   const size_t eb = dtype == PYR_BF16 ? 2 : 4;
   for (int i = 0; i < n_parts; ++i) {
@@ -613,7 +613,7 @@ pyr_status_t pyr_glue_linear_rows(const void* x, const void* w, const void* resi
   if (m == 0) return PYR_OK;
   const pyr::RowMap map = row_map(res_rows, n_src, n_dst, rows_stride);
   if (dtype == PYR_BF16 && pyr::gemm_tc_supported(x, w, residual, y, m, n, k))
-    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, nullptr, map, static_cast<cudaStream_t>(stream)));
+    PYR_GLUE(pyr::launch_gemm_tc(x, w, residual, y, m, n, k, pyr::glue_status_word(), map, static_cast<cudaStream_t>(stream)));
   PYR_GLUE(pyr::launch_glue_linear(x, w, residual, y, m, n, k, dtype, map, static_cast<cudaStream_t>(stream)));
 }
 pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* out, int64_t m, int32_t n,
@@ -622,7 +622,23 @@ pyr_status_t pyr_glue_linear_swiglu(const void* x, const void* w_gate, const voi
   if (m < 0 || n < 1 || k < 1) return PYR_ERR_INVALID;
   if (m == 0) return PYR_OK;
   if (dtype != PYR_BF16 || !pyr::gemm_tc_supported(x, w_gate, w_up, out, m, n, k)) return PYR_ERR_UNSUPPORTED;
-  PYR_GLUE(pyr::launch_gemm_tc_gated(x, w_gate, w_up, out, m, n, k, nullptr, static_cast<cudaStream_t>(stream)));
+  PYR_GLUE(pyr::launch_gemm_tc_gated(x, w_gate, w_up, out, m, n, k, pyr::glue_status_word(), static_cast<cudaStream_t>(stream)));
+}
+pyr_status_t pyr_glue_status(void* stream, int32_t* host_status) {
+  if (!host_status) return PYR_ERR_NULL;
+  int* word_dev = pyr::glue_status_word();
+  if (!word_dev) return PYR_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  const int zero = 0;
+  if (cudaMemcpyAsync(&word, word_dev, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return PYR_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return PYR_ERR_CUDA;
+  if (word != 0) {       // reported once, then the record starts clean
+    if (cudaMemcpyAsync(word_dev, &zero, sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess) return PYR_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return PYR_ERR_CUDA;
+  }
+  *host_status = word;
+  return word == 0 ? PYR_OK : PYR_ERR_TIMEOUT;
 }
 pyr_status_t pyr_glue_rope(void* x, const int32_t* pos, int64_t tokens, int32_t n_heads, int32_t head_dim,
                            int32_t dtype, void* stream) {

@@ -145,6 +145,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* w, const void* res, void* 
                            const RowMap& res_map, cudaStream_t s);
 cudaError_t launch_gemm_tc_gated(const void* x, const void* wg, const void* wu, void* out, int64_t M, int N, int K,
                                  int* status, cudaStream_t s);
+int* glue_status_word();     // the current GPU's status word of the glue GEMMs (null if it cannot be resolved)
 bool gemm_skinny_supported(const void* x, const void* w, const void* res, const void* y, int64_t M, int N, int K);
 // y may be given as up to four column parts ys[i] of [M, N / n_parts] each (n_parts > 1: no residual, parts of whole 128s)
 cudaError_t launch_gemm_skinny(const void* x, const void* w, const void* res, void* const* ys, int n_parts, int64_t M, int N,

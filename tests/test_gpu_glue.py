@@ -170,3 +170,13 @@ def test_split_linear_equals_separate_products(M, parts, part_n, K):
         scale = float(want.abs().max().clamp_min(1e-3))
         assert y.shape == (M, part_n)
         assert float((y.double() - want).abs().max()) <= 2 ** -7 * scale
+
+
+def test_glue_status_word_is_clean_after_the_linear_layers():
+    """pyr_glue_status: no bounded wait of a tensor-core linear layer ran out in this process; reading twice is fine."""
+    x = _r(300, 256, seed=71, dtype=torch.bfloat16)
+    w = (_r(512, 256, seed=72) * 0.05).to(torch.bfloat16)
+    pb.glue_linear(x, w)
+    pb.glue_linear(x[:8].contiguous(), w)
+    assert pb.glue_status() == 0
+    assert pb.glue_status() == 0

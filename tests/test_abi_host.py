@@ -209,6 +209,16 @@ def test_glue_entry_points_validate_before_any_launch():
     assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(2), i32(0), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_INVALID
     assert L.pyr_glue_linear_rows(P, P, NULL, P, i64(4), P, i32(2), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_ERR_NULL
     assert L.pyr_glue_linear_rows(P, P, P, P, i64(4), P, i32(0), i32(10), i32(4), i32(16), i32(16), i32(pb.PYR_F32), NULL) == pb.PYR_OK
+    # stacked projections: one to four parts, every part's pointer given
+    L.pyr_glue_linear_split.restype = L.pyr_glue_status.restype = C.c_int
+    two = (C.c_void_p * 2)(FAKE_DEV, FAKE_DEV)
+    hole = (C.c_void_p * 2)(FAKE_DEV, None)
+    assert L.pyr_glue_linear_split(P, P, None, i32(2), i64(4), i32(128), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear_split(P, P, hole, i32(2), i64(4), i32(128), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_NULL
+    assert L.pyr_glue_linear_split(P, P, two, i32(5), i64(4), i32(128), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_linear_split(P, P, two, i32(2), i64(4), i32(0), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_ERR_INVALID
+    assert L.pyr_glue_linear_split(P, P, two, i32(2), i64(0), i32(128), i32(64), i32(pb.PYR_BF16), NULL) == pb.PYR_OK
+    assert L.pyr_glue_status(NULL, None) == pb.PYR_ERR_NULL
 
 
 def test_select_first_flag_adds_the_inverse_list_to_the_plan():

@@ -170,3 +170,54 @@ def test_chained_stack_all_layers_batch2():
     cache.close()
     print(f"chained 7b stack, batch 2, 32 layers: {exact} sampled selections identical to the oracle's, "
           f"{ties} differ only within the 1e-6 tie band")
+
+
+@pytest.mark.parametrize("name,layers", [("13b_stack_32x4k", [1, 20, 39]), ("70b_gqa_16x8k", [1, 40])],
+                         ids=["13b_stack_32x4k", "70b_gqa_16x8k"])
+def test_full_size_select_first_against_oracle(name, layers):
+    """Select-first ordering at full size (the configuration bench.py times on the long per-head workloads):
+    kept sets under the tie rule, kept output rows on sampled rows, caches byte for byte."""
+    w = dict(synth.CONFIGS[name])
+    ratio = synth.ratio_schedule(w)
+    budgets = oracle.layer_budgets(w["prompt_len"], w["recent_len"], ratio)
+    B, Hq, Hkv, D, L, G = w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["recent_len"], w["sel_groups"]
+    rep = Hq // Hkv
+    per = Hq // G
+    for l in layers:
+        bud = budgets[l]
+        n, k, c = bud["n_in"], bud["k"], bud["c"]
+        cache = one_layer_cache(dict(w, max_new_tokens=0), n, k, flags=pb.PYR_FLAG_SELECT_FIRST)
+        Q, K, V = synth.stack_layer_inputs(w, l, n, device=DEV)
+        out = torch.empty_like(Q)
+        launches = pb.launch_count()
+        cache.prefill_layer(0, Q, K, V, out)
+        assert pb.launch_count() - launches == 5          # window tiles, score (2), selection, other tiles
+        n_out = cache.select_compact(0, K, V, out, per * D, out.stride(0), out.stride(1), per * D)
+        torch.cuda.synchronize()
+        assert cache.status() == 0 and n_out == bud["n_out"]
+        kept_all, _ = cache.kept(0)
+        Kc, Vc = cache.kv(0)
+        wts = oracle.recent_weights(L)
+        rng = np.random.default_rng(300 + l)
+        for (b, g) in _sample_pairs(B, G, 3, seed=50 + l):
+            heads = list(range(g * per, (g + 1) * per))
+            E = np.zeros((len(heads), c))
+            for hi, h in enumerate(heads):
+                A, _ = oracle.attention_weights(synth.widen(Q[b, :, h]), synth.widen(K[b, :, h // rep]),
+                                                oracle.softmax_scale_default(D), np.arange(c, n))
+                E[hi] = oracle.ensemble_score(A, L, wts)
+            kept = kept_all[b, g].cpu().numpy()
+            check_kept(kept, oracle.pooled_scores(E, 1)[0], k, n, L)
+            idx = torch.from_numpy(kept).to(DEV).long()
+            h = heads[int(rng.integers(len(heads)))]
+            js = np.sort(rng.choice(n_out, size=40, replace=False))
+            js[0], js[-1] = 0, n_out - 1                       # first kept row and the newest window row
+            A, _ = oracle.attention_weights(synth.widen(Q[b, :, h]), synth.widen(K[b, :, h // rep]),
+                                            oracle.softmax_scale_default(D), kept[js])
+            O_ref = A @ synth.widen(V[b, :, h // rep])
+            assert np.abs(synth.widen(out[b, torch.from_numpy(js).to(DEV), h]) - O_ref).max() <= 2e-2
+            assert torch.equal(Kc[b, h // rep, :n_out], K[b, idx, h // rep])
+            assert torch.equal(Vc[b, h // rep, :n_out], V[b, idx, h // rep])
+        cache.close()
+        del Q, K, V, out, cache
+        torch.cuda.empty_cache()

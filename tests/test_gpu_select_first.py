@@ -150,3 +150,28 @@ def test_select_first_with_reencoded_positions_and_generation_update():
     for l in range(2):
         assert torch.equal(s1[l][0], s0[l][0]) and torch.equal(s1[l][1], s0[l][1]) and s1[l][2] == s0[l][2]
         assert torch.equal(c1[l][0], c0[l][0]) and torch.equal(c1[l][1], c0[l][1])
+
+
+@pytest.mark.parametrize("dtype,D,flags", [("f32", 64, 0), ("bf16", 64, 0), ("bf16", 128, pb.PYR_FLAG_CUDA_CORE_PREFILL)],
+                         ids=["fp32", "bf16-d64", "bf16-cuda-core"])
+def test_select_first_falls_back_where_tensor_cores_do_not_apply(dtype, D, flags):
+    """With the flag set, configurations outside the tensor-core kernels take the default ordering: same launches,
+    same outputs, bit for bit."""
+    Hq, Hkv, G, B, n, L, k = 4, 2, 2, 2, 300, 64, 100
+    w = dict(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, sel_groups=G, dtype=dtype, batch=B,
+             prompt_len=n, recent_len=L, max_new_tokens=0, hitter_frac=0.05, hitter_mag=3.0)
+    Q, K, V = synth.stack_layer_inputs(w, 5, n, device=DEV, boost_queries=True)
+    res = []
+    for f in (flags | pb.PYR_FLAG_SELECT_FIRST, flags):
+        cache = one_layer_cache(w, n, k, flags=f)
+        out = torch.zeros_like(Q)
+        launches = pb.launch_count()
+        cache.prefill_layer(0, Q, K, V, out)
+        n_prefill = pb.launch_count() - launches
+        per = Hq // G
+        cache.select_compact(0, K, V, out, per * D, out.stride(0), out.stride(1), per * D)
+        torch.cuda.synchronize()
+        res.append((out.clone(), cache.kept(0)[0].clone(), n_prefill))
+        cache.close()
+    assert res[0][2] == res[1][2]
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])

@@ -229,3 +229,15 @@ def test_select_first_flag_adds_the_inverse_list_to_the_plan():
     b1, _ = pb.pyr_cache_bytes(flag_cfg)
     want = 2 * 4 * 512 * 4                     # B * G * N * 4 bytes
     assert b1 - b0 == (want + 255) // 256 * 256
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/pyr.h is the boundary: it must compile as C99 on its own (no C++ or CUDA types in the signatures)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "pyr.h"\nint main(void) { pyr_config_t c; (void)c; return (int)PYR_OK; }\n')
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                    "-I", os.path.join(ROOT, "include"), str(src)], check=True)

@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(GatherArgs a, int lanes_
 constexpr int kRowThreads = 256;
 constexpr int kRowUnroll = 4;
 
-__global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, int slab_lanes, int slabs, int items) {
+__global__ void __launch_bounds__(kRowThreads, 4) compact_rows_kernel(RowsArgs a, int slab_lanes, int slabs, int items) {
   // Items (one column slab of one stream) are dealt round-robin to a grid that fits the machine at
   // once: with one CTA per item a last, partly filled wave of CTAs would run at a fraction of the
   // bandwidth.
@@ -205,39 +205,54 @@ __global__ void __launch_bounds__(kRowThreads) compact_rows_kernel(RowsArgs a, i
   const int t = threadIdx.x;
   // Chunk i + 1 is read while chunk i is written: the sources of a later chunk lie above every
   // destination of an earlier one, so only the reads and writes of the same chunk need the barrier.
+  // (Four CTAs per SM: the few registers this costs in spills are cheaper than a CTA less.)
   uint4 buf[2][kRowUnroll];
-  int dst_row[2][kRowUnroll], ln[kRowUnroll];
+  int ln[kRowUnroll], rr[kRowUnroll];
 #pragma unroll
-  for (int u = 0; u < kRowUnroll; ++u) ln[u] = (u * kRowThreads + t) % lanes;
-  auto read_chunk = [&](int r0, uint4* bf, int* dr) {
-#pragma unroll
-    for (int u = 0; u < kRowUnroll; ++u) {
-      const int rr = (u * kRowThreads + t) / lanes;
-      dr[u] = -1;
-      if (rr < rows_per_iter && r0 + rr < a.n_out) {
-        const int src = idx[r0 + rr];
-        if (src != r0 + rr && src >= a.src_begin) {   // rows already in place are not touched
-          dr[u] = r0 + rr;
-          bf[u] = *reinterpret_cast<const uint4*>(base + (int64_t)src * row_bytes + ln[u] * 16);
-        }
-      }
-    }
-  };
-  auto write_chunk = [&](const uint4* bf, const int* dr) {
+  for (int u = 0; u < kRowUnroll; ++u) {
+    ln[u] = (u * kRowThreads + t) % lanes;
+    rr[u] = (u * kRowThreads + t) / lanes;
+  }
+  // The kept indices of a chunk are fetched one chunk before its rows are: the row loads then go out without
+  // first waiting for an index, and that wait was most of an iteration.
+  auto fetch_idx = [&](int r0, int* src) {
 #pragma unroll
     for (int u = 0; u < kRowUnroll; ++u)
-      if (dr[u] >= 0) *reinterpret_cast<uint4*>(base + (int64_t)dr[u] * row_bytes + ln[u] * 16) = bf[u];
+      src[u] = (rr[u] < rows_per_iter && r0 + rr[u] < a.n_out) ? idx[r0 + rr[u]] : -1;
+  };
+  // returns the mask of this thread's pieces that move (rows already in place are not touched)
+  auto read_chunk = [&](int r0, const int* src, uint4* bf) -> uint32_t {
+    uint32_t moved = 0;
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u) {
+      if (src[u] >= 0 && src[u] != r0 + rr[u] && src[u] >= a.src_begin) {
+        moved |= 1u << u;
+        bf[u] = *reinterpret_cast<const uint4*>(base + (int64_t)src[u] * row_bytes + ln[u] * 16);
+      }
+    }
+    return moved;
+  };
+  auto write_chunk = [&](int r0, const uint4* bf, uint32_t moved) {
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u)
+      if (moved & (1u << u)) *reinterpret_cast<uint4*>(base + (int64_t)(r0 + rr[u]) * row_bytes + ln[u] * 16) = bf[u];
   };
   const int first = a.dst_begin / rows_per_iter * rows_per_iter;
-  read_chunk(first, buf[0], dst_row[0]);
+  int src_a[kRowUnroll], src_b[kRowUnroll];
+  fetch_idx(first, src_a);
+  fetch_idx(first + rows_per_iter, src_b);
+  uint32_t mv0 = read_chunk(first, src_a, buf[0]), mv1 = 0;
   __syncthreads();
   for (int r0 = first; r0 < a.n_out; r0 += 2 * rows_per_iter) {
-    if (r0 + rows_per_iter < a.n_out) read_chunk(r0 + rows_per_iter, buf[1], dst_row[1]);
-    write_chunk(buf[0], dst_row[0]);
+    fetch_idx(r0 + 2 * rows_per_iter, src_a);
+    if (r0 + rows_per_iter < a.n_out) mv1 = read_chunk(r0 + rows_per_iter, src_b, buf[1]);
+    write_chunk(r0, buf[0], mv0);
     __syncthreads();
     if (r0 + rows_per_iter >= a.n_out) break;
-    if (r0 + 2 * rows_per_iter < a.n_out) read_chunk(r0 + 2 * rows_per_iter, buf[0], dst_row[0]);
-    write_chunk(buf[1], dst_row[1]);
+    fetch_idx(r0 + 3 * rows_per_iter, src_b);
+    mv0 = 0;
+    if (r0 + 2 * rows_per_iter < a.n_out) mv0 = read_chunk(r0 + 2 * rows_per_iter, src_a, buf[0]);
+    write_chunk(r0 + rows_per_iter, buf[1], mv1);
     __syncthreads();
   }
   }

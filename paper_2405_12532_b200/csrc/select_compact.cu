@@ -243,18 +243,33 @@ __global__ void __launch_bounds__(kRowThreads, 4) compact_rows_kernel(RowsArgs a
   fetch_idx(first + rows_per_iter, src_b);
   uint32_t mv0 = read_chunk(first, src_a, buf[0]), mv1 = 0;
   __syncthreads();
+  // The barrier after a chunk's write keeps a fast thread from writing rows a slow one has yet to read. Where every
+  // row moves up by at least d rows, a thread may run floor(d / rows per chunk) chunks ahead before that can happen,
+  // so the barrier is only taken every so many chunks (d never shrinks along a stream; it is read again at each
+  // barrier). Where rows barely move - the start of a stream - that is every chunk, as before.
+  int since = 0, every = 1;
+  auto barrier_if_due = [&](int r_next) {
+    if (++since >= every) {
+      __syncthreads();
+      since = 0;
+      const int at = r_next < a.n_out ? r_next : a.n_out - 1;
+      const int ahead = (idx[at] - at) / rows_per_iter;
+      every = ahead < 15 ? ahead + 1 : 16;
+    }
+  };
   for (int r0 = first; r0 < a.n_out; r0 += 2 * rows_per_iter) {
     fetch_idx(r0 + 2 * rows_per_iter, src_a);
     if (r0 + rows_per_iter < a.n_out) mv1 = read_chunk(r0 + rows_per_iter, src_b, buf[1]);
     write_chunk(r0, buf[0], mv0);
-    __syncthreads();
+    barrier_if_due(r0 + rows_per_iter);
     if (r0 + rows_per_iter >= a.n_out) break;
     fetch_idx(r0 + 3 * rows_per_iter, src_b);
     mv0 = 0;
     if (r0 + 2 * rows_per_iter < a.n_out) mv0 = read_chunk(r0 + 2 * rows_per_iter, src_a, buf[0]);
     write_chunk(r0 + rows_per_iter, buf[1], mv1);
-    __syncthreads();
+    barrier_if_due(r0 + 2 * rows_per_iter);
   }
+  __syncthreads();       // the next item starts from a barrier like the first
   }
 }
 
